@@ -1,0 +1,176 @@
+"""ctypes front end of the CPU oracle (``crisp_oracle.c``).
+
+Test infrastructure only: the tests, the smoke check and the benchmark's
+CPU-baseline leg load this; the CUDA library and its Python binding never do.
+The wrapper only allocates numpy arrays and forwards pointers.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "crisp_oracle.c")
+_LIB = os.path.join(_HERE, "libcrisp_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP for the row-parallel product)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                               "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+    return _lib
+
+
+def _p(a, t):
+    return a.ctypes.data_as(C.POINTER(t)) if a is not None else None
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def keep_count(k: int, block_k: int, keep_ratio: float):
+    nblk, kkeep = C.c_int(), C.c_int()
+    rc = lib().oracle_keep_count(C.c_int(k), C.c_int(block_k), C.c_double(keep_ratio),
+                                 C.byref(nblk), C.byref(kkeep))
+    if rc:
+        raise ValueError(f"oracle_keep_count rc={rc}")
+    return nblk.value, kkeep.value
+
+
+@dataclass
+class Mask:
+    rows: int
+    k: int
+    n: int
+    m: int
+    block_rows: int
+    block_k: int
+    kkeep: int
+    blk_col: np.ndarray   # int32 [nrt, kkeep]
+    nm_bits: np.ndarray   # uint32 [nrt*block_rows, ceil(nblk*block_k/32)]
+    score: np.ndarray     # uint64 [nrt, nblk]
+
+    @property
+    def nrt(self):
+        return (self.rows + self.block_rows - 1) // self.block_rows
+
+    @property
+    def nblk(self):
+        return (self.k + self.block_k - 1) // self.block_k
+
+    def dense(self) -> np.ndarray:
+        """Boolean [nrt*block_rows, nblk*block_k] view of the bit mask."""
+        bits = np.unpackbits(self.nm_bits.view(np.uint8), axis=1, bitorder="little")
+        return bits[:, : self.nblk * self.block_k].astype(bool)
+
+
+def build_mask(saliency: np.ndarray, n: int, m: int, block_rows: int, block_k: int,
+               keep_ratio: float | None = None, score_mode: int = 0, kkeep: int | None = None) -> Mask:
+    s = np.ascontiguousarray(saliency, dtype=np.float32)
+    rows, k = s.shape
+    nblk = (k + block_k - 1) // block_k
+    if kkeep is None:
+        nblk, kkeep = keep_count(k, block_k, keep_ratio)
+    nrt = (rows + block_rows - 1) // block_rows
+    wpr = (nblk * block_k + 31) // 32
+    blk_col = np.zeros((nrt, kkeep), dtype=np.int32)
+    nm_bits = np.zeros((nrt * block_rows, wpr), dtype=np.uint32)
+    score = np.zeros((nrt, nblk), dtype=np.uint64)
+    rc = lib().oracle_build_mask(_p(s, C.c_float), C.c_int64(s.strides[0] // 4), C.c_int(rows), C.c_int(k),
+                                 C.c_int(n), C.c_int(m), C.c_int(block_rows), C.c_int(block_k),
+                                 C.c_int(kkeep), C.c_int(score_mode),
+                                 _p(blk_col, C.c_int32), _p(nm_bits, C.c_uint32), _p(score, C.c_uint64))
+    if rc:
+        raise ValueError(f"oracle_build_mask rc={rc}")
+    return Mask(rows, k, n, m, block_rows, block_k, kkeep, blk_col, nm_bits, score)
+
+
+def encoded_sizes(rows, block_rows, block_k, n, m, kkeep):
+    nv, nw = C.c_int64(), C.c_int64()
+    rc = lib().oracle_encoded_sizes(C.c_int(rows), C.c_int(block_rows), C.c_int(block_k), C.c_int(n),
+                                    C.c_int(m), C.c_int(kkeep), C.byref(nv), C.byref(nw))
+    if rc:
+        raise ValueError(f"oracle_encoded_sizes rc={rc}")
+    return nv.value, nw.value
+
+
+def encode(w_bits: np.ndarray, mask: Mask):
+    """-> (vals uint16 [nvals], idx uint32 [nwords]) in the canonical order."""
+    w = np.ascontiguousarray(w_bits, dtype=np.uint16)
+    nv, nw = encoded_sizes(mask.rows, mask.block_rows, mask.block_k, mask.n, mask.m, mask.kkeep)
+    vals = np.zeros(nv, dtype=np.uint16)
+    idx = np.zeros(nw, dtype=np.uint32)
+    rc = lib().oracle_encode(_p(w, C.c_uint16), C.c_int64(w.strides[0] // 2), C.c_int(mask.rows), C.c_int(mask.k),
+                             C.c_int(mask.n), C.c_int(mask.m), C.c_int(mask.block_rows), C.c_int(mask.block_k),
+                             C.c_int(mask.kkeep), _p(np.ascontiguousarray(mask.blk_col), C.c_int32),
+                             _p(np.ascontiguousarray(mask.nm_bits), C.c_uint32),
+                             _p(vals, C.c_uint16), _p(idx, C.c_uint32))
+    if rc:
+        raise ValueError(f"oracle_encode rc={rc}")
+    return vals, idx
+
+
+def decode(blk_col, vals, idx, rows, k, n, m, block_rows, block_k, kkeep):
+    """-> (dense fp64 [rows, k], dense bf16 bits [rows, k])."""
+    wd = np.zeros((rows, k), dtype=np.float64)
+    wb = np.zeros((rows, k), dtype=np.uint16)
+    bc = np.ascontiguousarray(blk_col, dtype=np.int32)
+    rc = lib().oracle_decode(_p(bc, C.c_int32), _p(np.ascontiguousarray(vals, dtype=np.uint16), C.c_uint16),
+                             _p(np.ascontiguousarray(idx, dtype=np.uint32), C.c_uint32),
+                             C.c_int(rows), C.c_int(k), C.c_int(n), C.c_int(m), C.c_int(block_rows),
+                             C.c_int(block_k), C.c_int(kkeep), _p(wd, C.c_double), _p(wb, C.c_uint16))
+    if rc:
+        raise ValueError(f"oracle_decode rc={rc}")
+    return wd, wb
+
+
+def _spmm_call(fn, w_dense, x_bits):
+    wd = np.ascontiguousarray(w_dense, dtype=np.float64)
+    x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    rows, k = wd.shape
+    assert x.shape[0] == k
+    y = np.empty((rows, x.shape[1]), dtype=np.float64)
+    rc = fn(_p(wd, C.c_double), C.c_int(rows), C.c_int(k), _p(x, C.c_uint16),
+            C.c_int64(x.shape[1]), C.c_int64(x.shape[1]), _p(y, C.c_double))
+    if rc:
+        raise ValueError(f"oracle spmm rc={rc}")
+    return y
+
+
+def spmm_fp64(w_dense, x_bits):
+    """Y = Wd @ X by the literal fp64 triple loop."""
+    return _spmm_call(lib().oracle_spmm_fp64, w_dense, x_bits)
+
+
+def spmm_fp64_skipzero(w_dense, x_bits):
+    return _spmm_call(lib().oracle_spmm_fp64_skipzero, w_dense, x_bits)
+
+
+def spmm_fp64_rows(w_dense, x_bits, sel):
+    wd = np.ascontiguousarray(w_dense, dtype=np.float64)
+    x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    sel = np.ascontiguousarray(sel, dtype=np.int32)
+    rows, k = wd.shape
+    y = np.empty((len(sel), x.shape[1]), dtype=np.float64)
+    rc = lib().oracle_spmm_fp64_rows(_p(wd, C.c_double), C.c_int(rows), C.c_int(k), _p(x, C.c_uint16),
+                                     C.c_int64(x.shape[1]), C.c_int64(x.shape[1]),
+                                     _p(sel, C.c_int32), C.c_int(len(sel)), _p(y, C.c_double))
+    if rc:
+        raise ValueError(f"oracle_spmm_fp64_rows rc={rc}")
+    return y

@@ -1,0 +1,358 @@
+/*
+ * CPU oracle for the CRISP hybrid-sparsity path (test infrastructure only).
+ *
+ * Plain, slow, obviously-correct C.  It exists so that the CUDA library can be
+ * checked against something written independently from the paper; it shares no
+ * source, header, table or helper with the CUDA code and must never be called
+ * from the product path.  Only the tests, the smoke check and the CPU-baseline
+ * leg of the benchmark may load it.
+ *
+ * What it computes, in the paper's order:
+ *   - Algorithm 1 "apply fine-grained N:M pruning": per group of M consecutive
+ *     reduction elements keep the N of largest saliency            (Sec. III-A, III-C)
+ *   - Algorithm 1 "s_j = sum_i |T_w^i|": per-block score             (Sec. III-C)
+ *   - Algorithm 1 sort-per-row + select: the same number of blocks is kept in
+ *     every row of the block grid; the lowest-scored are pruned      (Sec. III-C)
+ *   - Algorithm 1 "f* = f (.) r": blocks keep their positions        (Sec. III-C)
+ *   - Sec. III-A storage: Blocked-ELLPACK column index per kept block and an
+ *     offset in [0, M) per kept value (zero-based, Sec. III-E worked example)
+ *   - Sec. III-E three-step sparse product, which equals the masked dense
+ *     product; the oracle is that definition: decode, then an fp64 triple loop.
+ *
+ * Readings where the paper is silent (mirrored in the design notes):
+ *   rows of W are output channels and groups/blocks run along the reduction
+ *   dimension; ties go to the lower index; saliency enters as |s| with NaN -> 0
+ *   and Inf -> FLT_MAX; the block score is an exact fixed-point integer sum so
+ *   that it does not depend on summation order; shapes are zero-padded to whole
+ *   blocks.
+ *
+ * All pointers are host memory.  bf16 values travel as uint16_t bit patterns.
+ * Every function returns 0 on success and a negative value on a bad argument.
+ */
+#include <float.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_SCORE_FRACTION_BITS 40
+
+/* ------------------------------------------------------------------ helpers */
+
+static double bf16_to_double(uint16_t b)
+{
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* |s| with the non-finite cases made orderable. */
+static float canonical_saliency(float s)
+{
+    if (isnan(s)) return 0.0f;
+    s = fabsf(s);
+    if (isinf(s)) return FLT_MAX;
+    return s;
+}
+
+static int log2_exact(int m)
+{
+    int b = 0;
+    while ((1 << b) < m) ++b;
+    return ((1 << b) == m) ? b : -1;
+}
+
+static int get_bit(const uint32_t *bits, int64_t words_per_row, int64_t row, int64_t col)
+{
+    return (int)((bits[row * words_per_row + (col >> 5)] >> (col & 31)) & 1u);
+}
+
+static void set_bit(uint32_t *bits, int64_t words_per_row, int64_t row, int64_t col)
+{
+    bits[row * words_per_row + (col >> 5)] |= (1u << (col & 31));
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------- shape bookkeeping */
+
+/* Blocks per row tile and how many of them survive: round-half-up of
+ * keep_ratio * nblk, evaluated in IEEE double. */
+int oracle_keep_count(int k, int block_k, double keep_ratio, int *nblk_out, int *kkeep_out)
+{
+    if (k <= 0 || block_k <= 0 || !(keep_ratio >= 0.0) || keep_ratio > 1.0) return -1;
+    int nblk = (k + block_k - 1) / block_k;
+    int kkeep = (int)floor(keep_ratio * (double)nblk + 0.5);
+    if (kkeep < 0) kkeep = 0;
+    if (kkeep > nblk) kkeep = nblk;
+    *nblk_out = nblk;
+    *kkeep_out = kkeep;
+    return 0;
+}
+
+/* ------------------------------------------------------------- mask build */
+
+/*
+ * saliency : [rows, k] fp32, leading dimension ld
+ * blk_col  : out, [nrt, kkeep] kept block columns per row tile, ascending
+ * nm_bits  : out, [nrt*block_rows, ceil(nblk*block_k/32)] uint32, bit (k & 31) of
+ *            word (k >> 5) of a row = 1 iff element (row, k) survives
+ * score    : out, optional (may be NULL), [nrt, nblk] fixed-point block scores
+ * score_mode 0: a block's score sums the saliency of its N:M survivors only
+ *               (Algorithm 1 prunes N:M first, so pruned weights contribute 0)
+ * score_mode 1: sums every element of the block
+ */
+int oracle_build_mask(const float *saliency, int64_t ld, int rows, int k,
+                      int n, int m, int block_rows, int block_k, int kkeep, int score_mode,
+                      int32_t *blk_col, uint32_t *nm_bits, uint64_t *score_out)
+{
+    if (!saliency || !nm_bits || rows <= 0 || k <= 0 || m <= 0 || n <= 0 || n > m) return -1;
+    if (block_rows <= 0 || block_k <= 0 || block_k % m != 0 || ld < k) return -1;
+    const int nrt = (rows + block_rows - 1) / block_rows;
+    const int nblk = (k + block_k - 1) / block_k;
+    if (kkeep < 0 || kkeep > nblk || (kkeep > 0 && !blk_col)) return -1;
+    const int64_t mp = (int64_t)nrt * block_rows;
+    const int64_t kp = (int64_t)nblk * block_k;
+    const int64_t wpr = (kp + 31) / 32;
+
+    /* step 1-2: padded, canonicalised saliency */
+    float *sp = (float *)calloc((size_t)(mp * kp), sizeof(float));
+    uint64_t *score = (uint64_t *)calloc((size_t)nrt * nblk, sizeof(uint64_t));
+    uint32_t *group_bits = (uint32_t *)calloc((size_t)(mp * wpr), sizeof(uint32_t));
+    if (!sp || !score || !group_bits) { free(sp); free(score); free(group_bits); return -2; }
+    float smax = 0.0f;
+    for (int r = 0; r < rows; ++r)
+        for (int c = 0; c < k; ++c) {
+            float v = canonical_saliency(saliency[(int64_t)r * ld + c]);
+            sp[(int64_t)r * kp + c] = v;
+            if (v > smax) smax = v;
+        }
+
+    /* step 3: N of M along k, largest saliency first, ties to the lower k */
+    int *order = (int *)malloc(sizeof(int) * (size_t)m);
+    for (int64_t r = 0; r < mp; ++r)
+        for (int64_t g = 0; g < kp / m; ++g) {
+            const float *v = sp + r * kp + g * m;
+            for (int i = 0; i < m; ++i) order[i] = i;
+            for (int i = 1; i < m; ++i) {              /* stable insertion sort, descending */
+                int cur = order[i], j = i - 1;
+                while (j >= 0 && v[order[j]] < v[cur]) { order[j + 1] = order[j]; --j; }
+                order[j + 1] = cur;
+            }
+            for (int i = 0; i < n; ++i) set_bit(group_bits, wpr, r, g * m + order[i]);
+        }
+    free(order);
+
+    /* step 4-5: fixed-point block scores  q(s) = floor(s * 2^(40 - e_max)) */
+    if (smax > 0.0f) {
+        const int e_max = ilogbf(smax);
+        for (int64_t r = 0; r < mp; ++r)
+            for (int64_t c = 0; c < kp; ++c) {
+                if (score_mode == 0 && !get_bit(group_bits, wpr, r, c)) continue;
+                double scaled = ldexp((double)sp[r * kp + c], ORACLE_SCORE_FRACTION_BITS - e_max);
+                score[(r / block_rows) * nblk + (c / block_k)] += (uint64_t)floor(scaled);
+            }
+    }
+
+    /* step 6-7: per row tile keep the kkeep best blocks (ties to the lower column) */
+    memset(nm_bits, 0, (size_t)(mp * wpr) * sizeof(uint32_t));
+    int *border = (int *)malloc(sizeof(int) * (size_t)nblk);
+    char *kept = (char *)malloc((size_t)nblk);
+    for (int rt = 0; rt < nrt; ++rt) {
+        const uint64_t *sc = score + (int64_t)rt * nblk;
+        for (int j = 0; j < nblk; ++j) border[j] = j;
+        for (int i = 1; i < nblk; ++i) {
+            int cur = border[i], j = i - 1;
+            while (j >= 0 && sc[border[j]] < sc[cur]) { border[j + 1] = border[j]; --j; }
+            border[j + 1] = cur;
+        }
+        memset(kept, 0, (size_t)nblk);
+        for (int i = 0; i < kkeep; ++i) kept[border[i]] = 1;
+        int slot = 0;
+        for (int j = 0; j < nblk; ++j) {
+            if (!kept[j]) continue;
+            blk_col[(int64_t)rt * kkeep + slot++] = j;
+            /* step 8: final mask = group bits AND block kept; positions unchanged */
+            for (int64_t r = (int64_t)rt * block_rows; r < (int64_t)(rt + 1) * block_rows; ++r)
+                for (int64_t c = (int64_t)j * block_k; c < (int64_t)(j + 1) * block_k; ++c)
+                    if (get_bit(group_bits, wpr, r, c)) set_bit(nm_bits, wpr, r, c);
+        }
+    }
+    if (score_out) memcpy(score_out, score, (size_t)nrt * nblk * sizeof(uint64_t));
+    free(border); free(kept); free(sp); free(score); free(group_bits);
+    return 0;
+}
+
+/* ------------------------------------------------------------ encode/decode */
+
+/* Number of stored values and of uint32 words of offset metadata. */
+int oracle_encoded_sizes(int rows, int block_rows, int block_k, int n, int m, int kkeep,
+                         int64_t *nvals, int64_t *nidx_words)
+{
+    int b = log2_exact(m);
+    if (b < 0 || rows <= 0) return -1;
+    int64_t nrt = (rows + block_rows - 1) / block_rows;
+    int64_t v = nrt * kkeep * block_rows * (block_k / m) * n;
+    *nvals = v;
+    *nidx_words = (v * b + 31) / 32;
+    return 0;
+}
+
+/*
+ * Canonical compressed format (Sec. III-A): for row tile rt, kept slot j, local
+ * row r, group g, v-th survivor of the group in ascending position:
+ *   vals[o] = W value, idx field o = its offset inside the M-vector (log2 M bits,
+ *   packed LSB-first into a uint32 stream), o = (((rt*kkeep+j)*block_rows+r)*G+g)*n+v.
+ * Elements in the zero padding are stored as 0x0000.
+ */
+int oracle_encode(const uint16_t *w, int64_t ld, int rows, int k,
+                  int n, int m, int block_rows, int block_k, int kkeep,
+                  const int32_t *blk_col, const uint32_t *nm_bits,
+                  uint16_t *vals, uint32_t *idx)
+{
+    const int b = log2_exact(m);
+    if (b < 0 || !w || !nm_bits || block_k % m != 0) return -1;
+    const int nrt = (rows + block_rows - 1) / block_rows;
+    const int nblk = (k + block_k - 1) / block_k;
+    const int64_t wpr = ((int64_t)nblk * block_k + 31) / 32;
+    const int groups = block_k / m;
+    int64_t nvals, nwords;
+    oracle_encoded_sizes(rows, block_rows, block_k, n, m, kkeep, &nvals, &nwords);
+    memset(idx, 0, (size_t)nwords * sizeof(uint32_t));
+    int64_t o = 0;
+    for (int rt = 0; rt < nrt; ++rt)
+        for (int j = 0; j < kkeep; ++j) {
+            const int jb = blk_col[(int64_t)rt * kkeep + j];
+            if (jb < 0 || jb >= nblk) return -3;
+            for (int r = 0; r < block_rows; ++r) {
+                const int64_t row = (int64_t)rt * block_rows + r;
+                for (int g = 0; g < groups; ++g) {
+                    int found = 0;
+                    for (int t = 0; t < m; ++t) {
+                        const int64_t col = (int64_t)jb * block_k + (int64_t)g * m + t;
+                        if (!get_bit(nm_bits, wpr, row, col)) continue;
+                        if (found == n) return -4;           /* more than N in a group */
+                        vals[o] = (row < rows && col < k) ? w[row * ld + col] : (uint16_t)0;
+                        const int64_t bit = o * b;
+                        for (int q = 0; q < b; ++q)
+                            if ((t >> q) & 1) idx[(bit + q) >> 5] |= 1u << ((bit + q) & 31);
+                        ++o; ++found;
+                    }
+                    if (found != n) return -4;               /* fewer than N in a group */
+                }
+            }
+        }
+    return (o == nvals) ? 0 : -5;
+}
+
+/* Inverse scatter into a zeroed dense [rows, k] matrix of doubles (and/or bf16 bits). */
+int oracle_decode(const int32_t *blk_col, const uint16_t *vals, const uint32_t *idx,
+                  int rows, int k, int n, int m, int block_rows, int block_k, int kkeep,
+                  double *w_dense, uint16_t *w_dense_bits)
+{
+    const int b = log2_exact(m);
+    if (b < 0) return -1;
+    const int nrt = (rows + block_rows - 1) / block_rows;
+    const int groups = block_k / m;
+    if (w_dense) memset(w_dense, 0, sizeof(double) * (size_t)rows * k);
+    if (w_dense_bits) memset(w_dense_bits, 0, sizeof(uint16_t) * (size_t)rows * k);
+    int64_t o = 0;
+    for (int rt = 0; rt < nrt; ++rt)
+        for (int j = 0; j < kkeep; ++j) {
+            const int jb = blk_col[(int64_t)rt * kkeep + j];
+            for (int r = 0; r < block_rows; ++r)
+                for (int g = 0; g < groups; ++g)
+                    for (int v = 0; v < n; ++v, ++o) {
+                        const int64_t bit = o * b;
+                        int t = 0;
+                        for (int q = 0; q < b; ++q)
+                            t |= (int)((idx[(bit + q) >> 5] >> ((bit + q) & 31)) & 1u) << q;
+                        const int64_t row = (int64_t)rt * block_rows + r;
+                        const int64_t col = (int64_t)jb * block_k + (int64_t)g * m + t;
+                        if (row >= rows || col >= k) {
+                            if (vals[o] != 0) return -6;     /* padding must hold zeros */
+                            continue;
+                        }
+                        if (w_dense) w_dense[row * k + col] = bf16_to_double(vals[o]);
+                        if (w_dense_bits) w_dense_bits[row * k + col] = vals[o];
+                    }
+        }
+    return 0;
+}
+
+/* ------------------------------------------------------------------- product */
+
+/*
+ * The three hardware steps of Sec. III-E compute exactly the masked dense product
+ *   Y[r, c] = sum_{t = 0}^{k-1} Wd[r, t] * X[t, c]
+ * so the oracle is this definition in fp64, a literal triple loop (threads split
+ * the rows of Y; each output is still one sequential sum over t).
+ */
+int oracle_spmm_fp64(const double *w_dense, int rows, int k,
+                     const uint16_t *x, int64_t ldx, int64_t ncols, double *y)
+{
+    if (!w_dense || !x || !y || ldx < ncols) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < ncols; ++c) {
+            double acc = 0.0;
+            for (int t = 0; t < k; ++t)
+                acc += w_dense[(int64_t)r * k + t] * bf16_to_double(x[(int64_t)t * ldx + c]);
+            y[(int64_t)r * ncols + c] = acc;
+        }
+    return 0;
+}
+
+/* Same definition for a chosen list of rows only: y is [nsel, ncols]. */
+int oracle_spmm_fp64_rows(const double *w_dense, int rows, int k,
+                          const uint16_t *x, int64_t ldx, int64_t ncols,
+                          const int32_t *sel, int nsel, double *y)
+{
+    if (!w_dense || !x || !y || !sel || ldx < ncols) return -1;
+    for (int i = 0; i < nsel; ++i) if (sel[i] < 0 || sel[i] >= rows) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int i = 0; i < nsel; ++i)
+        for (int64_t c = 0; c < ncols; ++c) {
+            double acc = 0.0;
+            for (int t = 0; t < k; ++t)
+                acc += w_dense[(int64_t)sel[i] * k + t] * bf16_to_double(x[(int64_t)t * ldx + c]);
+            y[(int64_t)i * ncols + c] = acc;
+        }
+    return 0;
+}
+
+/*
+ * Variant used only where the literal loop would take too long: for each row the
+ * t loop is outermost and terms with Wd == 0 are skipped.  Every Y[r, c] is still
+ * the sum over ascending t of the same products, so the result is identical up to
+ * the sign of zero; the tests show equality on small shapes.
+ */
+int oracle_spmm_fp64_skipzero(const double *w_dense, int rows, int k,
+                              const uint16_t *x, int64_t ldx, int64_t ncols, double *y)
+{
+    if (!w_dense || !x || !y || ldx < ncols) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < rows; ++r) {
+        double *yr = y + (int64_t)r * ncols;
+        for (int64_t c = 0; c < ncols; ++c) yr[c] = 0.0;
+        for (int t = 0; t < k; ++t) {
+            const double wv = w_dense[(int64_t)r * k + t];
+            if (wv == 0.0) continue;
+            const uint16_t *xr = x + (int64_t)t * ldx;
+            for (int64_t c = 0; c < ncols; ++c) yr[c] += wv * bf16_to_double(xr[c]);
+        }
+    }
+    return 0;
+}
