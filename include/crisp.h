@@ -1,0 +1,201 @@
+/*
+ * crisp.h - C ABI of libcrisp: CRISP hybrid structured sparsity on NVIDIA B200 (sm_100a).
+ *
+ * The library covers the inference-side hot path of the CRISP pruning framework
+ * (Aggarwal, Binici, Mitra: "CRISP: Hybrid Structured Sparsity for Class-aware Model
+ * Pruning"):
+ *
+ *   crisp_build_mask   saliency tensor -> hybrid mask: N of every M consecutive reduction
+ *                      elements (Sec. III-A; Algorithm 1, fine-grained N:M step) inside an
+ *                      equal number of kept coarse blocks per row of the block grid
+ *                      (Sec. III-A "uniform block pruning"; Algorithm 1, block score, per-row
+ *                      sort, select, prune).
+ *   crisp_encode       dense weight + mask -> compressed format: Blocked-ELLPACK column index
+ *                      per kept block and a log2(M)-bit offset per kept value (Sec. III-A),
+ *                      plus an execution image laid out for the tensor cores.
+ *   crisp_spmm         Y = W_hybrid * X, the three-step sparse product of Sec. III-E (load the
+ *                      activations of kept blocks, select activations by offset, multiply-
+ *                      accumulate), bf16 operands with fp32 accumulation.
+ *
+ * Conventions
+ *   - W is [rows, k]: rows are output channels, k = kernel_h * kernel_w * in_channels is the
+ *     reduction dimension and is contiguous.  N:M groups and coarse blocks run along k.
+ *   - A "row tile" is block_rows consecutive rows of W (one row of the paper's block grid).
+ *     nrt = ceil(rows / block_rows), nblk = ceil(k / block_k); shapes are zero-padded to
+ *     whole blocks (padded saliency and weights count as 0).
+ *   - X is [k, ncols] and Y is [rows, ncols], both row-major with ncols contiguous.
+ *   - bf16 values are passed as uint16_t bit patterns.
+ *   - Pointers named d_* are DEVICE memory owned by the caller; h_* are HOST memory owned by
+ *     the caller.  The library never allocates or frees device memory in the calls below:
+ *     the caller queries sizes, allocates, and keeps the buffers alive while the mask or
+ *     handle that refers to them is in use.  Device buffers must be 256-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All work is
+ *     enqueued on it and is asynchronous, except the *_export calls and
+ *     crisp_device_status, which synchronise the stream before returning.
+ *   - Every call returns a crisp_status_t.  Argument errors are detected on the host before
+ *     anything is launched.  No call throws, aborts or prints.
+ */
+#ifndef CRISP_H_
+#define CRISP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CRISP_API __attribute__((visibility("default")))
+#else
+#define CRISP_API
+#endif
+
+typedef enum {
+    CRISP_OK = 0,
+    CRISP_INVALID_ARG = 1,      /* null pointer, misaligned buffer, bad enum value            */
+    CRISP_UNSUPPORTED = 2,      /* pattern or size outside what the kernels implement         */
+    CRISP_BAD_SHAPE = 3,        /* non-positive extent, leading dimension too small           */
+    CRISP_BUFFER_TOO_SMALL = 4,
+    CRISP_CUDA_ERROR = 5,       /* a CUDA runtime/driver call or launch failed                */
+    CRISP_TIMEOUT = 6           /* a bounded wait inside a kernel expired (device status)     */
+} crisp_status_t;
+
+/* One pruned layer.  Sec. III-A: N:M sparsity inside B x B blocks (generalised here to
+ * block_rows x block_k). */
+typedef struct {
+    int32_t rows;        /* output channels, >= 1                                            */
+    int32_t k;           /* reduction length, >= 1                                           */
+    int32_t n;           /* kept elements per group, 1 <= n <= m                             */
+    int32_t m;           /* group length along k: 4 or 8                                     */
+    int32_t block_rows;  /* 32, 64 or 128                                                    */
+    int32_t block_k;     /* 32, 64, 96 or 128 (a multiple of 32 and of m)                    */
+    double  keep_ratio;  /* fraction of k-blocks kept in every row tile, in [0, 1]           */
+    int32_t score_mode;  /* 0: block score sums the N:M survivors (Algorithm 1 prunes N:M
+                            before it scores blocks); 1: sums every element of the block      */
+} crisp_layer_desc_t;
+
+typedef struct crisp_mask_s   *crisp_mask_t;    /* small host object, library-owned          */
+typedef struct crisp_handle_s *crisp_handle_t;  /* small host object, library-owned          */
+
+/* Roofline terms of one crisp_spmm call (bytes every algorithm must move, and multiply-
+ * accumulate counts), see crisp_bytes_model. */
+typedef struct {
+    int64_t nnz;              /* stored weight values, padding included                      */
+    int64_t vals_bytes;       /* 2 * nnz                                                     */
+    int64_t idx_bytes;        /* nnz * log2(m) / 8                                           */
+    int64_t blk_col_bytes;    /* 4 * nrt * kkeep                                             */
+    int64_t x_bytes;          /* rows of X under at least one kept block, read once          */
+    int64_t y_bytes;          /* rows * ncols * sizeof(Y element)                            */
+    int64_t useful_macs;      /* nnz * ncols                                                 */
+    int64_t slot_macs;        /* multiply-accumulate slots the chosen tensor-core path spends */
+    int32_t path;             /* which SpMM kernel the handle runs, see CRISP_PATH_*         */
+} crisp_bytes_t;
+
+#define CRISP_PATH_DIRECT 0   /* CUDA-core kernel on the canonical format (any shape)        */
+#define CRISP_PATH_DENSE  1   /* tcgen05 dense MMA over zero-expanded kept blocks            */
+#define CRISP_PATH_SPARSE 2   /* tcgen05 sparse (2:4) MMA over compressed kept blocks        */
+
+/* kkeep = floor(keep_ratio * nblk + 0.5), clamped to [0, nblk], evaluated in double on the
+ * host.  This is the "select by the current sparsity target" step of Algorithm 1 with the
+ * per-layer ratio given by the caller.  Error: INVALID_ARG / BAD_SHAPE / UNSUPPORTED. */
+CRISP_API crisp_status_t crisp_keep_count(const crisp_layer_desc_t *desc, int32_t *nblk, int32_t *kkeep);
+
+/* Bytes of the mask buffer (kept-block list + bit mask) and of the scratch workspace that
+ * crisp_build_mask needs for this layer. */
+CRISP_API crisp_status_t crisp_mask_sizes(const crisp_layer_desc_t *desc, size_t *mask_bytes,
+                                          size_t *workspace_bytes);
+
+/*
+ * Mask projection (Algorithm 1, N:M step, block score, per-row sort, select, prune).
+ *   d_saliency  [rows, k] fp32, leading dimension ld_s >= k (elements).  Sign is ignored;
+ *               NaN counts as 0, +-Inf as FLT_MAX.
+ *   d_mask_buf  out, mask_bytes; holds blk_col[nrt, kkeep] (int32, ascending per row tile)
+ *               and nm_bits[nrt*block_rows, nblk*block_k/32] (uint32, bit k%32 of word k/32).
+ *   d_workspace scratch, workspace_bytes; contents undefined afterwards.
+ *   out         receives a mask object that refers to d_mask_buf (not to d_saliency or
+ *               d_workspace).  Free it with crisp_mask_destroy.
+ * Steps: per group of m elements keep the n largest |s| (ties: lower k); block score =
+ * exact fixed-point sum of floor(|s| * 2^(40 - e_max)), e_max = exponent of the largest |s|
+ * in the layer; per row tile keep the kkeep highest scores (ties: lower column); final bit =
+ * group bit AND block kept.  Blocks keep their positions (no column permutation).
+ */
+CRISP_API crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s,
+                                          const crisp_layer_desc_t *desc,
+                                          void *d_mask_buf, void *d_workspace, void *stream,
+                                          crisp_mask_t *out);
+
+/* Copy the mask to host: h_blk_col [nrt*kkeep] int32, h_nm_bits [nrt*block_rows *
+ * nblk*block_k/32] uint32.  Either may be NULL.  Synchronises `stream`. */
+CRISP_API crisp_status_t crisp_mask_export(crisp_mask_t mask, int32_t *h_blk_col, uint32_t *h_nm_bits,
+                                           void *stream);
+
+/* Shape bookkeeping of a mask (any out pointer may be NULL). */
+CRISP_API crisp_status_t crisp_mask_info(crisp_mask_t mask, crisp_layer_desc_t *desc, int32_t *nrt,
+                                         int32_t *nblk, int32_t *kkeep);
+
+/* Bytes of the canonical compressed format and of the execution image for this mask. */
+CRISP_API crisp_status_t crisp_encode_sizes(crisp_mask_t mask, size_t *canonical_bytes,
+                                            size_t *exec_bytes);
+
+/*
+ * Compress (Sec. III-A storage format; Algorithm 1 "f* = f (.) r").
+ *   d_w_bf16        [rows, k] bf16, leading dimension ld_w >= k
+ *   d_canonical_buf out: blk_col[nrt*kkeep] int32 | vals[nnz] bf16 | idx[ceil(nnz*b/32)] uint32
+ *                   with b = log2(m).  Order of values: row tile, kept slot, local row,
+ *                   group, value (ascending position); idx field o occupies bits
+ *                   [o*b, o*b+b) of the uint32 stream, LSB first; offsets are zero-based
+ *                   positions inside the m-vector (Sec. III-E example).  Values in the zero
+ *                   padding are stored as 0.
+ *   d_exec_buf      out: tensor-core-ready copy used by crisp_spmm (opaque) + status word.
+ *   out             handle referring to both buffers (not to d_w_bf16 nor to the mask).
+ */
+CRISP_API crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t mask,
+                                      void *d_canonical_buf, void *d_exec_buf, void *stream,
+                                      crisp_handle_t *out);
+
+/* Element counts of the canonical arrays (for sizing the host buffers of crisp_export). */
+CRISP_API crisp_status_t crisp_encoded_counts(crisp_handle_t h, int64_t *n_blk_col, int64_t *n_vals,
+                                              int64_t *n_idx_words);
+
+/* Copy the canonical format to host (any pointer may be NULL).  Synchronises `stream`. */
+CRISP_API crisp_status_t crisp_export(crisp_handle_t h, int32_t *h_blk_col, uint16_t *h_vals,
+                                      uint32_t *h_idx, void *stream);
+
+/* Inverse of crisp_encode: scatter into a dense [rows, k] bf16 matrix (zeros elsewhere). */
+CRISP_API crisp_status_t crisp_decode(crisp_handle_t h, uint16_t *d_w_dense_bf16, int64_t ld,
+                                      void *stream);
+
+/*
+ * Y = W_hybrid * X (Sec. III-E, steps 1-3).
+ *   d_x_bf16 [k, ncols] bf16, leading dimension ldx >= ncols
+ *   d_y      [rows, ncols], leading dimension ldy >= ncols, bf16 (y_dtype 0, round to
+ *            nearest even from the fp32 accumulator) or fp32 (y_dtype 1)
+ * Rows of X under blocks that no row tile kept are never read.  A layer with kkeep = 0
+ * yields Y = 0.  The tensor-core kernels need X and Y 16-byte aligned with ldx*2 and
+ * ldy*sizeof(element) multiples of 16; other layouts run on the direct kernel.
+ */
+CRISP_API crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ldx,
+                                    int64_t ncols, void *d_y, int64_t ldy, int32_t y_dtype, void *stream);
+
+/* Restrict crisp_spmm of this handle to one kernel family (CRISP_PATH_*), or -1 for the
+ * default choice.  UNSUPPORTED if the handle's execution image cannot serve that path. */
+CRISP_API crisp_status_t crisp_set_path(crisp_handle_t h, int32_t path);
+
+/* Read the device status word of the handle (0 = no kernel reported a problem; otherwise a
+ * crisp_status_t, e.g. CRISP_TIMEOUT when a bounded wait expired).  Synchronises `stream`. */
+CRISP_API crisp_status_t crisp_device_status(crisp_handle_t h, void *stream, int32_t *status_out);
+
+/* Algorithmic byte and multiply-accumulate counts of one crisp_spmm(ncols) call.  Reads the
+ * kept-block list back with a blocking copy (not for use inside a timed region). */
+CRISP_API crisp_status_t crisp_bytes_model(crisp_handle_t h, int64_t ncols, int32_t y_dtype,
+                                           crisp_bytes_t *out);
+
+CRISP_API void crisp_mask_destroy(crisp_mask_t mask);
+CRISP_API void crisp_destroy(crisp_handle_t h);
+CRISP_API const char *crisp_status_string(crisp_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CRISP_H_ */

@@ -1,0 +1,307 @@
+"""ctypes binding of libcrisp's C ABI (see include/crisp.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of
+``libcrisp.so``.  PyTorch supplies device buffers and streams.  There is no CPU or
+PyTorch fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcrisp.so")
+
+OK, INVALID_ARG, UNSUPPORTED, BAD_SHAPE, BUFFER_TOO_SMALL, CUDA_ERROR, TIMEOUT = range(7)
+PATH_DIRECT, PATH_DENSE, PATH_SPARSE = 0, 1, 2
+PATH_NAMES = {0: "direct", 1: "dense_tcgen05", 2: "sparse_tcgen05"}
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("rows", C.c_int32), ("k", C.c_int32), ("n", C.c_int32), ("m", C.c_int32),
+                ("block_rows", C.c_int32), ("block_k", C.c_int32), ("keep_ratio", C.c_double),
+                ("score_mode", C.c_int32)]
+
+
+class BytesModel(C.Structure):
+    _fields_ = [("nnz", C.c_int64), ("vals_bytes", C.c_int64), ("idx_bytes", C.c_int64),
+                ("blk_col_bytes", C.c_int64), ("x_bytes", C.c_int64), ("y_bytes", C.c_int64),
+                ("useful_macs", C.c_int64), ("slot_macs", C.c_int64), ("path", C.c_int32)]
+
+    def as_dict(self):
+        return {f: int(getattr(self, f)) for f, _ in self._fields_}
+
+
+class CrispError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = crisp_status_string(code) if _lib is not None else str(code)
+        super().__init__(f"{where}: {msg} (status {code})")
+
+
+_lib = None
+
+
+def load(path: Optional[str] = None):
+    """Load libcrisp.so (built in-tree by ``paper_2311_14272_b200.build``)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(
+            f"{p} not found: build it with `python -m paper_2311_14272_b200.build` "
+            "(there is no fallback implementation)")
+    lib = C.CDLL(p)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    P = C.POINTER
+    sig = {
+        "crisp_keep_count": [P(LayerDesc), P(i32), P(i32)],
+        "crisp_mask_sizes": [P(LayerDesc), P(sz), P(sz)],
+        "crisp_build_mask": [vp, i64, P(LayerDesc), vp, vp, vp, P(vp)],
+        "crisp_mask_export": [vp, vp, vp, vp],
+        "crisp_mask_info": [vp, P(LayerDesc), P(i32), P(i32), P(i32)],
+        "crisp_encode_sizes": [vp, P(sz), P(sz)],
+        "crisp_encode": [vp, i64, vp, vp, vp, vp, P(vp)],
+        "crisp_encoded_counts": [vp, P(i64), P(i64), P(i64)],
+        "crisp_export": [vp, vp, vp, vp, vp],
+        "crisp_decode": [vp, vp, i64, vp],
+        "crisp_spmm": [vp, vp, i64, i64, vp, i64, i32, vp],
+        "crisp_set_path": [vp, i32],
+        "crisp_device_status": [vp, vp, P(i32)],
+        "crisp_bytes_model": [vp, i64, i32, P(BytesModel)],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    lib.crisp_mask_destroy.argtypes = [vp]
+    lib.crisp_mask_destroy.restype = None
+    lib.crisp_destroy.argtypes = [vp]
+    lib.crisp_destroy.restype = None
+    lib.crisp_status_string.argtypes = [C.c_int]
+    lib.crisp_status_string.restype = C.c_char_p
+    _lib = lib
+    return lib
+
+
+def crisp_status_string(code: int) -> str:
+    return load().crisp_status_string(code).decode()
+
+
+status_string = crisp_status_string
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise CrispError(code, where)
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor / numpy array / int."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def make_desc(rows, k, n, m, block_rows, block_k, keep_ratio, score_mode=0) -> LayerDesc:
+    return LayerDesc(rows, k, n, m, block_rows, block_k, float(keep_ratio), score_mode)
+
+
+# ------------------------------------------------------------------ raw entry points
+
+def crisp_keep_count(desc: LayerDesc):
+    nblk, kkeep = C.c_int32(), C.c_int32()
+    _check(load().crisp_keep_count(C.byref(desc), C.byref(nblk), C.byref(kkeep)), "crisp_keep_count")
+    return nblk.value, kkeep.value
+
+
+def crisp_mask_sizes(desc: LayerDesc):
+    a, b = C.c_size_t(), C.c_size_t()
+    _check(load().crisp_mask_sizes(C.byref(desc), C.byref(a), C.byref(b)), "crisp_mask_sizes")
+    return a.value, b.value
+
+
+def crisp_build_mask(d_saliency, ld_s: int, desc: LayerDesc, d_mask_buf, d_workspace, stream=None) -> int:
+    out = C.c_void_p()
+    _check(load().crisp_build_mask(_ptr(d_saliency), ld_s, C.byref(desc), _ptr(d_mask_buf), _ptr(d_workspace),
+                                   _stream(stream), C.byref(out)), "crisp_build_mask")
+    return out.value
+
+
+def crisp_mask_info(mask: int):
+    d, a, b, c = LayerDesc(), C.c_int32(), C.c_int32(), C.c_int32()
+    _check(load().crisp_mask_info(mask, C.byref(d), C.byref(a), C.byref(b), C.byref(c)), "crisp_mask_info")
+    return d, a.value, b.value, c.value
+
+
+def crisp_mask_export(mask: int, h_blk_col, h_nm_bits, stream=None):
+    _check(load().crisp_mask_export(mask, _ptr(h_blk_col), _ptr(h_nm_bits), _stream(stream)), "crisp_mask_export")
+
+
+def crisp_encode_sizes(mask: int):
+    a, b = C.c_size_t(), C.c_size_t()
+    _check(load().crisp_encode_sizes(mask, C.byref(a), C.byref(b)), "crisp_encode_sizes")
+    return a.value, b.value
+
+
+def crisp_encode(d_w, ld_w: int, mask: int, d_canonical, d_exec, stream=None) -> int:
+    out = C.c_void_p()
+    _check(load().crisp_encode(_ptr(d_w), ld_w, mask, _ptr(d_canonical), _ptr(d_exec), _stream(stream),
+                               C.byref(out)), "crisp_encode")
+    return out.value
+
+
+def crisp_encoded_counts(handle: int):
+    a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(load().crisp_encoded_counts(handle, C.byref(a), C.byref(b), C.byref(c)), "crisp_encoded_counts")
+    return a.value, b.value, c.value
+
+
+def crisp_export(handle: int, h_blk_col, h_vals, h_idx, stream=None):
+    _check(load().crisp_export(handle, _ptr(h_blk_col), _ptr(h_vals), _ptr(h_idx), _stream(stream)), "crisp_export")
+
+
+def crisp_decode(handle: int, d_w_dense, ld: int, stream=None):
+    _check(load().crisp_decode(handle, _ptr(d_w_dense), ld, _stream(stream)), "crisp_decode")
+
+
+def crisp_spmm(handle: int, d_x, ldx: int, ncols: int, d_y, ldy: int, y_dtype: int = 0, stream=None):
+    _check(load().crisp_spmm(handle, _ptr(d_x), ldx, ncols, _ptr(d_y), ldy, y_dtype, _stream(stream)), "crisp_spmm")
+
+
+def crisp_set_path(handle: int, path: int):
+    _check(load().crisp_set_path(handle, path), "crisp_set_path")
+
+
+def crisp_device_status(handle: int, stream=None) -> int:
+    s = C.c_int32()
+    _check(load().crisp_device_status(handle, _stream(stream), C.byref(s)), "crisp_device_status")
+    return s.value
+
+
+def crisp_bytes_model(handle: int, ncols: int, y_dtype: int = 0) -> dict:
+    b = BytesModel()
+    _check(load().crisp_bytes_model(handle, ncols, y_dtype, C.byref(b)), "crisp_bytes_model")
+    return b.as_dict()
+
+
+def crisp_mask_destroy(mask: int):
+    if mask:
+        load().crisp_mask_destroy(mask)
+
+
+def crisp_destroy(handle: int):
+    if handle:
+        load().crisp_destroy(handle)
+
+
+# -------------------------------------------------- buffer-owning convenience wrapper
+
+class HybridLayer:
+    """Owns the device buffers of one pruned layer and forwards to the C ABI.
+
+    ``build_mask`` -> ``encode`` -> ``spmm`` mirror crisp_build_mask / crisp_encode /
+    crisp_spmm; tensors are torch CUDA tensors (bf16 tensors or their int16/uint16 views).
+    """
+
+    def __init__(self, rows, k, n, m, block_rows, block_k, keep_ratio, score_mode=0, device="cuda"):
+        import torch
+        self.torch = torch
+        self.device = torch.device(device)
+        self.desc = make_desc(rows, k, n, m, block_rows, block_k, keep_ratio, score_mode)
+        self.nblk, self.kkeep = crisp_keep_count(self.desc)
+        self.nrt = (rows + block_rows - 1) // block_rows
+        mask_bytes, ws_bytes = crisp_mask_sizes(self.desc)
+        self.mask_buf = torch.empty(mask_bytes, dtype=torch.uint8, device=self.device)
+        self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=self.device)
+        self.mask = 0
+        self.handle = 0
+        self.canonical_buf = None
+        self.exec_buf = None
+
+    def build_mask(self, saliency, stream=None):
+        assert saliency.is_cuda and saliency.dtype == self.torch.float32 and saliency.stride(1) == 1
+        crisp_mask_destroy(self.mask)
+        self.mask = crisp_build_mask(saliency, saliency.stride(0), self.desc, self.mask_buf, self.workspace, stream)
+        return self
+
+    def export_mask(self, stream=None):
+        import numpy as np
+        wpr = self.nblk * self.desc.block_k // 32
+        blk_col = np.zeros((self.nrt, self.kkeep), dtype=np.int32)
+        nm_bits = np.zeros((self.nrt * self.desc.block_rows, wpr), dtype=np.uint32)
+        crisp_mask_export(self.mask, blk_col, nm_bits, stream)
+        return blk_col, nm_bits
+
+    def encode(self, w, stream=None):
+        assert w.is_cuda and w.element_size() == 2 and w.stride(1) == 1
+        torch = self.torch
+        cbytes, ebytes = crisp_encode_sizes(self.mask)
+        if self.canonical_buf is None or self.canonical_buf.numel() < cbytes:
+            self.canonical_buf = torch.empty(cbytes, dtype=torch.uint8, device=self.device)
+        if self.exec_buf is None or self.exec_buf.numel() < ebytes:
+            self.exec_buf = torch.empty(ebytes, dtype=torch.uint8, device=self.device)
+        crisp_destroy(self.handle)
+        self.handle = crisp_encode(w, w.stride(0), self.mask, self.canonical_buf, self.exec_buf, stream)
+        return self
+
+    def export(self, stream=None):
+        import numpy as np
+        nb, nv, nw = crisp_encoded_counts(self.handle)
+        blk_col = np.zeros(nb, dtype=np.int32)
+        vals = np.zeros(nv, dtype=np.uint16)
+        idx = np.zeros(nw, dtype=np.uint32)
+        crisp_export(self.handle, blk_col, vals, idx, stream)
+        return blk_col.reshape(self.nrt, self.kkeep), vals, idx
+
+    def decode(self, stream=None):
+        torch = self.torch
+        w = torch.empty((self.desc.rows, self.desc.k), dtype=torch.bfloat16, device=self.device)
+        crisp_decode(self.handle, w, w.stride(0), stream)
+        return w
+
+    def spmm(self, x, y=None, y_dtype=0, stream=None):
+        torch = self.torch
+        assert x.is_cuda and x.element_size() == 2 and x.stride(1) == 1 and x.shape[0] == self.desc.k
+        ncols = x.shape[1]
+        if y is None:
+            y = torch.empty((self.desc.rows, ncols), dtype=torch.float32 if y_dtype else torch.bfloat16,
+                            device=self.device)
+        crisp_spmm(self.handle, x, x.stride(0), ncols, y, y.stride(0), y_dtype, stream)
+        return y
+
+    def set_path(self, path: int):
+        crisp_set_path(self.handle, path)
+
+    def device_status(self, stream=None) -> int:
+        return crisp_device_status(self.handle, stream)
+
+    def bytes_model(self, ncols, y_dtype=0):
+        return crisp_bytes_model(self.handle, ncols, y_dtype)
+
+    def close(self):
+        crisp_destroy(self.handle)
+        crisp_mask_destroy(self.mask)
+        self.handle = 0
+        self.mask = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

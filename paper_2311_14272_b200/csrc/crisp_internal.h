@@ -1,0 +1,74 @@
+// Internal declarations shared by the translation units of libcrisp.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "crisp.h"
+
+namespace crisp {
+
+// Shape of one layer after padding to whole blocks.
+struct Geometry {
+    int rows, k, n, m, bm, bk;
+    int score_mode;
+    int nrt;        // row tiles
+    int nblk;       // k-blocks per row tile
+    int kkeep;      // kept k-blocks per row tile
+    int wpr;        // uint32 words of bit mask per (padded) row = nblk * bk / 32
+    int idx_bits;   // log2(m)
+    __host__ __device__ int64_t mp() const { return (int64_t)nrt * bm; }
+    __host__ __device__ int64_t kp() const { return (int64_t)nblk * bk; }
+    __host__ __device__ int groups() const { return bk / m; }
+    __host__ __device__ int64_t vals_per_block() const { return (int64_t)bm * groups() * n; }
+    __host__ __device__ int64_t nnz() const { return (int64_t)nrt * kkeep * vals_per_block(); }
+    __host__ __device__ int64_t idx_words() const { return (nnz() * idx_bits + 31) / 32; }
+};
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+}  // namespace crisp
+
+struct crisp_mask_s {
+    crisp::Geometry g;
+    int32_t *d_blk_col;     // [nrt, kkeep]
+    uint32_t *d_nm_bits;    // [mp, wpr]
+};
+
+struct crisp_handle_s {
+    crisp::Geometry g;
+    // canonical format
+    int32_t *d_blk_col;
+    uint16_t *d_vals;
+    uint32_t *d_idx;
+    // execution image
+    int32_t *d_status;      // first word of the exec buffer
+    uint8_t *d_exec;        // payload after the 256-byte header
+    size_t exec_payload_bytes;
+    int exec_kind;          // CRISP_PATH_* the image was laid out for (DIRECT = none)
+    int forced_path;        // -1 = default
+};
+
+namespace crisp {
+
+// mask_kernels.cu
+cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, int32_t *d_blk_col,
+                              uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes,
+                              cudaStream_t st);
+size_t mask_workspace_bytes(const Geometry &g);
+
+// encode_kernels.cu
+cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geometry &g,
+                                    const int32_t *d_mask_blk_col, const uint32_t *d_nm_bits,
+                                    int32_t *d_blk_col, uint16_t *d_vals, uint32_t *d_idx,
+                                    cudaStream_t st);
+cudaError_t launch_decode(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
+                          const uint32_t *d_idx, uint16_t *d_w, int64_t ld, cudaStream_t st);
+
+// spmm_direct.cu
+cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
+                               const uint32_t *d_idx, const uint16_t *d_x, int64_t ldx, int64_t ncols,
+                               void *d_y, int64_t ldy, int y_dtype, cudaStream_t st);
+
+}  // namespace crisp

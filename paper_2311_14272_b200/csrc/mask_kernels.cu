@@ -1,0 +1,230 @@
+// Mask projection kernels: saliency -> hybrid (block + N:M) mask.
+//
+// Algorithm 1 of the paper, restricted to one layer with the block keep count given:
+//   K-M0  layer-wide maximum of the canonical saliency (sets the fixed-point scale)
+//   K-M1  per group of M: keep the N largest (fine-grained N:M step) and accumulate the
+//         block scores s_j = sum |T_w| as exact fixed-point integers
+//   K-M2  per row of the block grid: keep the kkeep highest-scored blocks and clear the
+//         bits of the pruned ones (blocks keep their positions)
+// All three stream the data once with coalesced 32-byte-per-lane accesses; the work is
+// bound by HBM bandwidth (one compare network per 4 bytes read).
+#include "crisp_internal.h"
+
+namespace crisp {
+
+namespace {
+
+constexpr int kScoreFractionBits = 40;
+constexpr int kM1Threads = 256;
+constexpr int kM1ChunkK = 256;           // k-elements covered by one warp pass (32 lanes x 8)
+
+// |s| as an order-preserving uint32 key: NaN -> 0, Inf -> FLT_MAX.
+__device__ __forceinline__ uint32_t canonical_key(float s) {
+    uint32_t u = __float_as_uint(s) & 0x7FFFFFFFu;
+    if (u > 0x7F800000u) return 0u;
+    if (u == 0x7F800000u) return 0x7F7FFFFFu;
+    return u;
+}
+
+// Eight consecutive saliency values of one row, zero beyond the matrix.
+__device__ __forceinline__ void load8(const float *__restrict__ s, int64_t ld, int rows, int k,
+                                      int64_t row, int64_t k0, bool vec_ok, uint32_t key[8]) {
+    if (row >= rows || k0 >= k) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) key[i] = 0u;
+        return;
+    }
+    const float *p = s + row * ld + k0;
+    if (vec_ok && k0 + 8 <= k) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(p));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+        key[0] = canonical_key(a.x); key[1] = canonical_key(a.y);
+        key[2] = canonical_key(a.z); key[3] = canonical_key(a.w);
+        key[4] = canonical_key(b.x); key[5] = canonical_key(b.y);
+        key[6] = canonical_key(b.z); key[7] = canonical_key(b.w);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) key[i] = (k0 + i < k) ? canonical_key(__ldg(p + i)) : 0u;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+max_key_kernel(const float *__restrict__ s, int64_t ld, int rows, int k, bool vec_ok,
+               uint32_t *__restrict__ max_key) {
+    const int chunks = (k + 7) / 8;
+    const int64_t total = (int64_t)rows * chunks;
+    uint32_t best = 0u;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / chunks;
+        const int64_t k0 = (i - row * chunks) * 8;
+        uint32_t key[8];
+        load8(s, ld, rows, k, row, k0, vec_ok, key);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) best = max(best, key[j]);
+    }
+    best = __reduce_max_sync(0xFFFFFFFFu, best);
+    if ((threadIdx.x & 31) == 0 && best) atomicMax(max_key, best);
+}
+
+// Exponent of a positive finite float given by its bits (ilogb), denormals included.
+__device__ __forceinline__ int key_exponent(uint32_t key) {
+    const int e = (int)(key >> 23);
+    return e ? e - 127 : (31 - __clz(key)) - 149;
+}
+
+// Bit i of the result is set iff element i is among the N largest of its group of M
+// (ties to the lower index).  M is 4 or 8; the 8 keys hold two groups or one.
+template <int M>
+__device__ __forceinline__ uint32_t top_n_bits(const uint32_t key[8], int n) {
+    uint32_t bits = 0u;
+#pragma unroll
+    for (int g = 0; g < 8 / M; ++g) {
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            int rank = 0;
+#pragma unroll
+            for (int j = 0; j < M; ++j) {
+                const uint32_t a = key[g * M + j], b = key[g * M + i];
+                rank += (a > b) || (a == b && j < i);
+            }
+            bits |= (rank < n ? 1u : 0u) << (g * M + i);
+        }
+    }
+    return bits;
+}
+
+// One CTA covers bm rows x 256 k-elements.  Warp w takes rows w, w+8, ...; lane l owns the 8
+// elements at k = chunk*256 + 8*l of each of its rows, so every lane stays inside one block
+// column and keeps its partial block score in a register.
+template <int M>
+__global__ void __launch_bounds__(kM1Threads)
+group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_ok,
+                    const uint32_t *__restrict__ max_key, uint32_t *__restrict__ nm_bits,
+                    unsigned long long *__restrict__ score) {
+    __shared__ unsigned long long s_score[kM1ChunkK / 32 + 2];
+    const int rt = blockIdx.y;
+    const int chunk = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t k0 = (int64_t)chunk * kM1ChunkK + lane * 8;
+    const int first_blk = (chunk * kM1ChunkK) / g.bk;
+    if (threadIdx.x < kM1ChunkK / 32 + 2) s_score[threadIdx.x] = 0ull;
+    __syncthreads();
+
+    const uint32_t mk = *max_key;
+    const double scale = mk ? ldexp(1.0, kScoreFractionBits - key_exponent(mk)) : 0.0;
+    const bool in_kp = k0 < g.kp();
+    unsigned long long acc = 0ull;
+    for (int r = warp; r < g.bm; r += kM1Threads / 32) {
+        const int64_t row = (int64_t)rt * g.bm + r;
+        uint32_t key[8];
+        load8(s, ld, g.rows, g.k, row, k0, vec_ok, key);
+        const uint32_t bits = top_n_bits<M>(key, g.n);
+        const uint32_t counted = g.score_mode == 0 ? bits : 0xFFu;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if ((counted >> i) & 1u)
+                acc += __double2ull_rd((double)__uint_as_float(key[i]) * scale);
+        // four lanes assemble one 32-bit mask word
+        uint32_t word = bits << (8 * (lane & 3));
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+        if ((lane & 3) == 0 && in_kp) nm_bits[row * g.wpr + (k0 >> 5)] = word;
+    }
+    if (in_kp && acc) atomicAdd(&s_score[(int)(k0 / g.bk) - first_blk], acc);
+    __syncthreads();
+    if (threadIdx.x < kM1ChunkK / 32 + 2) {
+        const int jb = first_blk + threadIdx.x;
+        const unsigned long long v = s_score[threadIdx.x];
+        if (jb < g.nblk && v) atomicAdd(&score[(int64_t)rt * g.nblk + jb], v);
+    }
+}
+
+// One CTA per row tile: rank the block scores, emit the kept columns in ascending order and
+// clear the mask words of pruned blocks.
+__global__ void __launch_bounds__(256)
+block_select_kernel(Geometry g, const unsigned long long *__restrict__ score,
+                    int32_t *__restrict__ blk_col, uint32_t *__restrict__ nm_bits) {
+    extern __shared__ unsigned long long sm[];
+    unsigned long long *sc = sm;                                   // [nblk]
+    int *kept = reinterpret_cast<int *>(sm + g.nblk);              // [nblk]
+    __shared__ int s_warp_tot[8];
+    __shared__ int s_base;
+    const int rt = blockIdx.x;
+    for (int j = threadIdx.x; j < g.nblk; j += blockDim.x) sc[j] = score[(int64_t)rt * g.nblk + j];
+    if (threadIdx.x == 0) s_base = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < g.nblk; j += blockDim.x) {
+        const unsigned long long mine = sc[j];
+        int rank = 0;
+        for (int t = 0; t < g.nblk; ++t) {
+            const unsigned long long o = sc[t];
+            rank += (o > mine) || (o == mine && t < j);
+        }
+        kept[j] = rank < g.kkeep;
+    }
+    __syncthreads();
+    // ascending compaction: block-wide exclusive scan over chunks of blockDim.x flags
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int j0 = 0; j0 < g.nblk; j0 += blockDim.x) {
+        const int j = j0 + threadIdx.x;
+        const int f = (j < g.nblk) ? kept[j] : 0;
+        const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, f);
+        const int before = __popc(ballot & ((1u << lane) - 1u));
+        if (lane == 0) s_warp_tot[warp] = __popc(ballot);
+        __syncthreads();
+        int warp_off = 0, tot = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+            if (w < warp) warp_off += s_warp_tot[w];
+            tot += s_warp_tot[w];
+        }
+        if (f) blk_col[(int64_t)rt * g.kkeep + s_base + warp_off + before] = j;
+        __syncthreads();
+        if (threadIdx.x == 0) s_base += tot;
+        __syncthreads();
+    }
+    // final mask = group bits AND block kept
+    const int wpb = g.bk / 32;
+    const int64_t items = (int64_t)g.nblk * g.bm * wpb;
+    for (int64_t i = threadIdx.x; i < items; i += blockDim.x) {
+        const int w = (int)(i % wpb);
+        const int r = (int)((i / wpb) % g.bm);
+        const int jb = (int)(i / ((int64_t)wpb * g.bm));
+        if (!kept[jb]) nm_bits[((int64_t)rt * g.bm + r) * g.wpr + jb * wpb + w] = 0u;
+    }
+}
+
+}  // namespace
+
+// workspace: [0] max key (uint32), padded to 256 B; then score[nrt * nblk] uint64.
+size_t mask_workspace_bytes(const Geometry &g) {
+    return kAlign + align_up((size_t)g.nrt * g.nblk * sizeof(unsigned long long));
+}
+
+cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, int32_t *d_blk_col,
+                              uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes,
+                              cudaStream_t st) {
+    uint32_t *max_key = reinterpret_cast<uint32_t *>(d_workspace);
+    unsigned long long *score =
+        reinterpret_cast<unsigned long long *>(reinterpret_cast<uint8_t *>(d_workspace) + kAlign);
+    cudaError_t e = cudaMemsetAsync(d_workspace, 0, workspace_bytes, st);
+    if (e != cudaSuccess) return e;
+    const bool vec_ok = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_s) & 15u) == 0);
+
+    const int64_t items = (int64_t)g.rows * ((g.k + 7) / 8);
+    int grid0 = (int)((items + 255) / 256 < 148 * 8 ? (items + 255) / 256 : 148 * 8);
+    if (grid0 < 1) grid0 = 1;
+    max_key_kernel<<<grid0, 256, 0, st>>>(d_s, ld, g.rows, g.k, vec_ok, max_key);
+
+    dim3 grid1((unsigned)((g.kp() + kM1ChunkK - 1) / kM1ChunkK), (unsigned)g.nrt);
+    if (g.m == 4)
+        group_select_kernel<4><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
+    else
+        group_select_kernel<8><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
+
+    const size_t smem = (size_t)g.nblk * (sizeof(unsigned long long) + sizeof(int));
+    block_select_kernel<<<g.nrt, 256, smem, st>>>(g, score, d_blk_col, d_nm_bits);
+    return cudaGetLastError();
+}
+
+}  // namespace crisp

@@ -1,0 +1,180 @@
+"""CUDA path against the CPU oracle, through the C ABI, on the same seeded inputs.
+
+Masks and encodings must match bit for bit; the product must satisfy
+max |Y - Yref| <= 1e-2 * (1 + |Yref|) and ||Y - Yref||_F / ||Yref||_F <= 5e-3."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2311_14272_b200 import workloads as wl
+
+from helpers import (assert_mask_and_encoding_equal, bf16_dev, check_tolerance, gpu_layer,
+                     oracle_layer, to_dev, y_to_f64)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2311_14272_b200 import binding as B
+    B.load()
+    assert torch.cuda.is_available()
+    return B, torch
+
+
+def rand_inputs(rows, k, ncols, seed, relu=False):
+    rng = np.random.default_rng(seed)
+    w = wl.f32_to_bf16_bits((rng.standard_normal((rows, k)) * 0.05).astype(np.float32))
+    s = (np.abs(wl.bf16_bits_to_f32(w)) * rng.uniform(0.5, 1.5, (rows, k))).astype(np.float32)
+    x = rng.standard_normal((k, ncols)).astype(np.float32)
+    if relu:
+        x = np.maximum(x, 0)
+    return w, s, wl.f32_to_bf16_bits(x)
+
+
+CASES = [
+    # rows, k, ncols, n, m, bm, bk, keep   (several tiles and a ragged tail in every dimension)
+    (256, 1024, 512, 2, 4, 32, 64, 0.5),
+    (200, 576, 333, 1, 4, 64, 64, 0.25),
+    (96, 144, 1000, 2, 8, 32, 32, 0.5),
+    (24, 27, 130, 2, 4, 64, 64, 1.0),
+    (70, 200, 77, 3, 4, 32, 32, 0.4),
+    (300, 640, 520, 4, 8, 128, 64, 0.75),
+    (260, 512, 264, 1, 8, 128, 64, 0.5),
+    (64, 96, 50, 8, 8, 32, 32, 0.67),
+    (130, 384, 96, 2, 4, 128, 128, 0.34),
+    (64, 288, 40, 3, 8, 64, 96, 0.67),
+]
+
+
+@pytest.mark.parametrize("rows,k,ncols,n,m,bm,bk,keep", CASES)
+@pytest.mark.parametrize("y_dtype", [0, 1])
+def test_layer_matches_oracle(env, rows, k, ncols, n, m, bm, bk, keep, y_dtype):
+    B, torch = env
+    w, s, x = rand_inputs(rows, k, ncols, seed=rows + k + ncols)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
+    L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    dec = L.decode().view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(dec, wb)
+    y = L.spmm(bf16_dev(x, torch), y_dtype=y_dtype)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    check_tolerance(y_to_f64(y, torch), oracle.spmm_fp64(wd, x))
+    L.close()
+
+
+def test_score_mode_all_elements(env):
+    B, torch = env
+    w, _, x = rand_inputs(128, 512, 64, seed=77)
+    # odd block columns: one dominant element per group; even ones: four medium elements, so the
+    # survivor sum and the all-element sum rank the blocks differently
+    rng = np.random.default_rng(3)
+    s = rng.uniform(0.9, 1.1, (128, 512)).astype(np.float32)
+    odd = ((np.arange(512) // 64) % 2 == 1)
+    s[:, odd & (np.arange(512) % 4 != 0)] *= np.float32(0.01)
+    s[:, odd & (np.arange(512) % 4 == 0)] *= np.float32(1.5)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, 1, 4, 32, 64, 0.5, score_mode=1)
+    mk0 = oracle.build_mask(s, 1, 4, 32, 64, 0.5, score_mode=0)
+    assert not np.array_equal(mk.blk_col, mk0.blk_col)       # the two readings differ on this input
+    L = gpu_layer(B, torch, w, s, 1, 4, 32, 64, 0.5, score_mode=1)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    L0 = gpu_layer(B, torch, w, s, 1, 4, 32, 64, 0.5, score_mode=0)
+    v0, i0 = oracle.encode(w, mk0)
+    assert_mask_and_encoding_equal(L0, mk0, v0, i0)
+
+
+def test_padded_leading_dimensions_and_odd_alignment(env):
+    B, torch = env
+    w, s, x = rand_inputs(100, 250, 90, seed=5)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, 2, 4, 32, 64, 0.5)
+    L = gpu_layer(B, torch, w, s, 2, 4, 32, 64, 0.5, ld_pad=3)       # ld = 253: scalar-load path
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    xbuf = torch.zeros((250, 97), dtype=torch.bfloat16, device="cuda")
+    xbuf[:, :90] = bf16_dev(x, torch)
+    ybuf = torch.full((100, 101), 7.0, dtype=torch.bfloat16, device="cuda")
+    L.spmm(xbuf[:, :90], y=ybuf[:, :90])
+    check_tolerance(y_to_f64(ybuf[:, :90], torch), oracle.spmm_fp64(wd, x))
+    assert torch.all(ybuf[:, 90:] == 7.0)                                # nothing written past ncols
+
+
+def test_non_finite_negative_and_tied_saliency(env):
+    B, torch = env
+    rng = np.random.default_rng(11)
+    rows, k = 64, 256
+    w = wl.f32_to_bf16_bits(rng.standard_normal((rows, k)).astype(np.float32))
+    s = rng.integers(0, 4, (rows, k)).astype(np.float32)               # many ties, many zeros
+    s[rng.random((rows, k)) < 0.05] = np.nan
+    s[rng.random((rows, k)) < 0.02] = np.inf
+    s[rng.random((rows, k)) < 0.02] = -np.inf
+    s *= np.where(rng.random((rows, k)) < 0.5, -1, 1).astype(np.float32)
+    for (n, m) in [(2, 4), (3, 8)]:
+        mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, 32, 32, 0.5)
+        L = gpu_layer(B, torch, w, s, n, m, 32, 32, 0.5)
+        assert_mask_and_encoding_equal(L, mk, vals, idx)
+    # all-zero saliency: every score ties at 0 -> first blocks, first n of every group
+    z = np.zeros((rows, k), dtype=np.float32)
+    mk, vals, idx, wd, wb = oracle_layer(w, z, 2, 4, 32, 32, 0.25)
+    L = gpu_layer(B, torch, w, z, 2, 4, 32, 32, 0.25)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    # denormal-only saliency still ranks correctly
+    d = (rng.integers(1, 1000, (rows, k)) * 1.4e-45).astype(np.float32)
+    mk, vals, idx, wd, wb = oracle_layer(w, d, 1, 4, 32, 32, 0.5)
+    L = gpu_layer(B, torch, w, d, 1, 4, 32, 32, 0.5)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+
+
+def test_no_kept_block_writes_zeros(env):
+    B, torch = env
+    w, s, x = rand_inputs(64, 27, 50, seed=2)
+    L = gpu_layer(B, torch, w, s, 2, 4, 64, 64, 0.4)
+    assert L.kkeep == 0
+    y = torch.full((64, 50), 3.0, dtype=torch.bfloat16, device="cuda")
+    L.spmm(bf16_dev(x, torch), y=y)
+    assert torch.count_nonzero(y).item() == 0
+    assert L.export()[1].size == 0
+
+
+@pytest.mark.parametrize("n,m,bm,bk,keep", [(2, 4, 32, 64, 0.5), (1, 8, 64, 32, 0.25), (4, 8, 128, 64, 1.0)])
+def test_identity_activation_is_bit_exact(env, n, m, bm, bk, keep):
+    """X = I: every output is a single product by 1, exact in fp32 and in bf16, so Y must equal
+    the decoded weight bit for bit; this pins every index and offset path."""
+    B, torch = env
+    rows, k = 192, 256
+    w, s, _ = rand_inputs(rows, k, 8, seed=n * 10 + m)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
+    L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
+    eye = torch.eye(k, dtype=torch.bfloat16, device="cuda")
+    y = L.spmm(eye)
+    got = y.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got & 0x7FFF, wb & 0x7FFF)                      # (sign of zero aside)
+    assert np.array_equal(wl.bf16_bits_to_f32(got), wl.bf16_bits_to_f32(wb))
+    assert np.array_equal(y_to_f64(y, torch), oracle.spmm_fp64(wd, wl.f32_to_bf16_bits(np.eye(k, dtype=np.float32))))
+
+
+def test_config1_full(env):
+    B, torch = env
+    l = wl.config1()[0]
+    w, s, x = wl.make_layer_inputs(l)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, l.n, l.m, l.block_rows, l.block_k, l.keep_ratio)
+    L = gpu_layer(B, torch, w, s, l.n, l.m, l.block_rows, l.block_k, l.keep_ratio)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    y = L.spmm(bf16_dev(x, torch))
+    check_tolerance(y_to_f64(y, torch), oracle.spmm_fp64(wd, x))
+
+
+def test_config2_full(env):
+    B, torch = env
+    l = wl.config2()[0]
+    w, s, x = wl.make_layer_inputs(l)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, l.n, l.m, l.block_rows, l.block_k, l.keep_ratio)
+    assert mk.kkeep == 9
+    L = gpu_layer(B, torch, w, s, l.n, l.m, l.block_rows, l.block_k, l.keep_ratio)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    y = L.spmm(bf16_dev(x, torch))
+    sel = np.array([0, 63, 64, 100, 255], dtype=np.int32)
+    ref_rows = oracle.spmm_fp64_rows(wd, x, sel)                          # the literal definition
+    full = oracle.spmm_fp64_skipzero(wd, x)                               # shown equal on small shapes
+    assert np.array_equal(full[sel], ref_rows)
+    check_tolerance(y_to_f64(y, torch), full)
