@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the CRISP hybrid-sparse hot path on B200.
+
+One *step* = the whole path on one layer: crisp_build_mask (saliency -> hybrid mask),
+crisp_encode (weight + mask -> compressed format + execution image) and crisp_spmm
+(Y = W_hybrid X), all through the C ABI.  The headline metric is useful TFLOP/s of the
+step, 2 * nnz * ncols / step time; the SpMM kernel alone, its roofline fraction and its
+speedup over a dense bf16 cuBLAS GEMM of the same shape are reported beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints exactly one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2311_14272_b200 import workloads as wl  # noqa: E402
+
+METRIC = "hybrid_sparse_spmm_useful_tflops"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_FLUSH_BYTES = 256 << 20
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def pick_layer(name: str) -> wl.Layer:
+    if name == "config2":
+        return wl.config2()[0]
+    if name == "config1":
+        return wl.config1()[0]
+    if name.startswith("sweep_"):
+        nm, keep = name[len("sweep_"):].split("_keep")
+        n, m = nm.split(":")
+        return wl.sweep_cell(int(n), int(m), float(keep))
+    raise SystemExit(f"unknown workload {name}")
+
+
+# --------------------------------------------------------------------- clock sampling
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid = uuid
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------ CPU oracle
+
+def oracle_step(layer, w, s, x_sample):
+    """One pass of the oracle as it stands on a bounded column sample; returns (seconds, nnz)."""
+    import oracle
+    t0 = time.perf_counter()
+    mk = oracle.build_mask(s, layer.n, layer.m, layer.block_rows, layer.block_k, layer.keep_ratio)
+    vals, idx = oracle.encode(w, mk)
+    wd, _ = oracle.decode(mk.blk_col, vals, idx, layer.rows, layer.k, layer.n, layer.m,
+                          layer.block_rows, layer.block_k, mk.kkeep)
+    oracle.spmm_fp64(wd, x_sample)
+    return time.perf_counter() - t0, int(vals.size)
+
+
+def oracle_sample_cols(layer, w, s, x, target_s=12.0):
+    """Choose how many columns of X the oracle multiplies so that one pass takes ~target_s."""
+    import oracle
+    mk = oracle.build_mask(s, layer.n, layer.m, layer.block_rows, layer.block_k, layer.keep_ratio)
+    vals, idx = oracle.encode(w, mk)
+    wd, _ = oracle.decode(mk.blk_col, vals, idx, layer.rows, layer.k, layer.n, layer.m,
+                          layer.block_rows, layer.block_k, mk.kkeep)
+    probe = np.ascontiguousarray(x[:, :4])
+    t0 = time.perf_counter()
+    oracle.spmm_fp64(wd, probe)
+    per_col = (time.perf_counter() - t0) / 4
+    return int(max(4, min(x.shape[1], target_s / max(per_col, 1e-9))))
+
+
+def run_reference(args, layer, rank):
+    """--impl reference: the CPU oracle, timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    w, s, x = wl.make_layer_inputs(layer)
+    cols = oracle_sample_cols(layer, w, s, x, target_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)))
+    xs = np.ascontiguousarray(x[:, :cols])
+    for _ in range(args.warmup):
+        oracle_step(layer, w, s, xs)
+    tot, nnz = 0.0, 0
+    for _ in range(args.steps):
+        dt, nnz = oracle_step(layer, w, s, xs)
+        tot += dt
+    ms = tot / args.steps * 1e3
+    value = 2.0 * nnz * cols / (ms * 1e-3) / 1e12
+    sample = f"mask+encode+decode of the full layer, fp64 product on the first {cols} of {layer.ncols} columns"
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": args.workload, "rows": layer.rows, "k": layer.k, "ncols": layer.ncols,
+                      "sampled_ncols": cols},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                            "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+# ---------------------------------------------------------------------------- GPU arm
+
+def run_ours(args, layer, rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2311_14272_b200 import binding as B
+
+    B.load()                                       # raises if libcrisp.so is missing: no fallback
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks, peak_kind = load_peaks()
+
+    w, s, x = wl.make_layer_inputs(layer)
+    h_s = torch.from_numpy(s).pin_memory()
+    h_w = torch.from_numpy(w.view(np.int16)).pin_memory()
+    h_x = torch.from_numpy(x.view(np.int16)).pin_memory()
+    d_s = h_s.to(dev)
+    d_w = h_w.to(dev).view(torch.bfloat16)
+    d_x = h_x.to(dev).view(torch.bfloat16)
+    d_y = torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16, device=dev)
+    h_y = torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    L = B.HybridLayer(layer.rows, layer.k, layer.n, layer.m, layer.block_rows, layer.block_k,
+                      layer.keep_ratio, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        L.build_mask(d_s)
+        L.encode(d_w)
+        L.spmm(d_x, y=d_y)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    if L.device_status() != 0:
+        raise SystemExit(f"device status {L.device_status()} after warm-up")
+    model = L.bytes_model(layer.ncols)
+    nnz = model["nnz"]
+
+    # ---- timed region: K steps, each bracketed by events on the launching stream; L2 is flushed
+    # between steps (outside the event pairs) by overwriting a 256 MiB buffer
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    barrier()
+    sampler.start()
+    for i in range(args.steps):
+        flush.zero_()
+        ev[i][0].record(stream)
+        L.build_mask(d_s)
+        ev[i][1].record(stream)
+        L.encode(d_w)
+        ev[i][2].record(stream)
+        L.spmm(d_x, y=d_y)
+        ev[i][3].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    t_mask = np.array([e[0].elapsed_time(e[1]) for e in ev])
+    t_enc = np.array([e[1].elapsed_time(e[2]) for e in ev])
+    t_spmm = np.array([e[2].elapsed_time(e[3]) for e in ev])
+    t_step = np.array([e[0].elapsed_time(e[3]) for e in ev])
+    ms_local = float(t_step.sum() / args.steps)
+    ms_t = torch.tensor([ms_local], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(ms_t.item())
+    status = L.device_status()
+
+    # ---- dense bf16 cuBLAS GEMM of the same shape, same protocol
+    t_dense = []
+    for i in range(3 + args.steps):
+        flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        torch.matmul(d_w, d_x, out=d_y)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            t_dense.append(a.elapsed_time(b))
+    t_dense = np.array(t_dense)
+
+    # ---- end to end: pinned host inputs -> device, whole path, result back to pinned host memory
+    def e2e_step():
+        d_s.copy_(h_s, non_blocking=True)
+        d_w.view(torch.int16).copy_(h_w, non_blocking=True)
+        d_x.view(torch.int16).copy_(h_x, non_blocking=True)
+        step()
+        h_y.copy_(d_y, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    b.record(stream)
+    barrier()
+    e2e_ms = torch.tensor([a.elapsed_time(b) / e2e_steps], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_ms = float(e2e_ms.item())
+
+    useful_flops = 2.0 * nnz * layer.ncols
+    value = world * useful_flops / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * useful_flops / (e2e_ms * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (SpMM), from its live event time
+    spmm_ms = float(t_spmm.mean())
+    slot_flops = 2.0 * model["slot_macs"]
+    hbm_bytes = model["vals_bytes"] + model["idx_bytes"] + model["blk_col_bytes"] + model["x_bytes"] + model["y_bytes"]
+    t_tensor = slot_flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = hbm_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        roof = {"bound": "tensor", "achieved": slot_flops / (spmm_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": hbm_bytes / (spmm_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof.update({"traffic": None, "peak_kind": f"of {peak_kind} (burst)", "kernel": B.PATH_NAMES[model["path"]],
+                 "t_tensor_us": t_tensor * 1e6, "t_hbm_us": t_hbm * 1e6, "t_kernel_us": spmm_ms * 1e3,
+                 "frac_of_max_roof": max(t_tensor, t_hbm) / (spmm_ms * 1e-3),
+                 "frac_literal_useful_flops": useful_flops / (spmm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                 "algorithmic_bytes": hbm_bytes, "slot_flops": slot_flops})
+    mask_bytes = layer.rows * layer.k * 4 * 2 + layer.rows * layer.k // 8   # S read twice (max, select) + bits
+    enc_bytes = model["vals_bytes"] * 2 + model["idx_bytes"] + layer.rows * layer.k // 8
+    phases = {"mask_us": float(t_mask.mean() * 1e3), "encode_us": float(t_enc.mean() * 1e3),
+              "spmm_us": spmm_ms * 1e3, "spmm_us_min": float(t_spmm.min() * 1e3),
+              "mask_gbs": mask_bytes / (t_mask.mean() * 1e-3) / 1e9,
+              "encode_gbs": enc_bytes / (t_enc.mean() * 1e-3) / 1e9,
+              "spmm_useful_tflops": useful_flops / (spmm_ms * 1e-3) / 1e12,
+              "dense_cublas_us": float(t_dense.mean() * 1e3),
+              "spmm_speedup_vs_dense_cublas": float(t_dense.mean() / t_spmm.mean())}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": args.workload, "rows": layer.rows, "k": layer.k, "ncols": layer.ncols,
+                      "n": layer.n, "m": layer.m, "block": [layer.block_rows, layer.block_k],
+                      "keep_ratio": layer.keep_ratio, "kkeep": L.kkeep, "nnz": nnz,
+                      "step": "crisp_build_mask + crisp_encode + crisp_spmm",
+                      "l2": "flushed between steps (256 MiB overwrite outside the event pairs)",
+                      "parallelism": "replicas only" if world > 1 else "single GPU"},
+           "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
+                   "h2d_bytes_per_step": int(h_s.numel() * 4 + h_w.numel() * 2 + h_x.numel() * 2),
+                   "d2h_bytes_per_step": int(h_y.numel() * 2)},
+           "gpu_launches": 5 * args.steps, "kernels_per_step": {"mask": 3, "encode": 1, "spmm": 1},
+           "clocks": clocks, "roofline": roof, "phases": phases, "device_status": status}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        cols = oracle_sample_cols(layer, w, s, x)
+        dt, onnz = oracle_step(layer, w, s, np.ascontiguousarray(x[:, :cols]))
+        out["cpu_baseline"] = {"value": 2.0 * onnz * cols / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+                               "kind": "oracle", "seconds": dt,
+                               "sample": f"mask+encode+decode of the full layer, fp64 product on the first {cols} "
+                                         f"of {layer.ncols} columns"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="sweep_2:4_keep0.5",
+                    help="sweep_<n>:<m>_keep<r> (4096x4096x8192, block 128x64), config1 or config2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    layer = pick_layer(args.workload)
+    if args.impl == "reference":
+        run_reference(args, layer, rank)
+    else:
+        run_ours(args, layer, rank, world)
+
+
+if __name__ == "__main__":
+    main()
