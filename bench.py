@@ -129,10 +129,11 @@ def oracle_sample_cols(layer, w, s, x, target_s=12.0):
     vals, idx = oracle.encode(w, mk)
     wd, _ = oracle.decode(mk.blk_col, vals, idx, layer.rows, layer.k, layer.n, layer.m,
                           layer.block_rows, layer.block_k, mk.kkeep)
-    probe = np.ascontiguousarray(x[:, :4])
+    pc = min(256, x.shape[1])
+    probe = np.ascontiguousarray(x[:, :pc])
     t0 = time.perf_counter()
     oracle.spmm_fp64(wd, probe)
-    per_col = (time.perf_counter() - t0) / 4
+    per_col = (time.perf_counter() - t0) / pc
     return int(max(4, min(x.shape[1], target_s / max(per_col, 1e-9))))
 
 
