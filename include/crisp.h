@@ -125,6 +125,34 @@ CRISP_API crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s,
                                           void *d_mask_buf, void *d_workspace, void *stream,
                                           crisp_mask_t *out);
 
+/*
+ * Same result as crisp_build_mask, for callers that cannot hand over a scratch workspace
+ * because they are not allowed to allocate device memory at the point of the call (a plug-in
+ * inside a framework that owns all device memory, a loop that must stay allocation-free after
+ * start-up, a process whose pool is fully committed).  The paper has no counterpart of this
+ * call; it is a packaging variant of the mask projection.
+ *
+ * The scratch lives in a fixed array of CRISP_STATIC_SCRATCH_BYTES inside the library image;
+ * every GPU that loads the library holds it until the process exits.  The call allocates and
+ * frees nothing, on host-visible CUDA APIs or otherwise.  Inputs and outputs are still the
+ * caller's: d_saliency, d_mask_buf (crisp_mask_sizes gives its size) and the returned mask.
+ *
+ * Limits and rules
+ *   - The layer's workspace (256 bytes + 8 bytes per coarse block, i.e. per (row tile,
+ *     k-block) pair) must fit: at most 32736 coarse blocks.  Larger layers are refused with
+ *     CRISP_BUFFER_TOO_SMALL before anything is launched; use crisp_build_mask for them.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call during set-up, before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps what the last call wrote.  Each
+ *     call clears it on `stream` before use, so calls issued one after another on the same
+ *     stream are safe; calls that may run concurrently on the GPU (different streams or host
+ *     threads without ordering between them) race on it and give wrong masks.
+ */
+#define CRISP_STATIC_SCRATCH_BYTES (256 * 1024)
+CRISP_API crisp_status_t crisp_build_mask_static(const float *d_saliency, int64_t ld_s,
+                                                 const crisp_layer_desc_t *desc, void *d_mask_buf,
+                                                 void *stream, crisp_mask_t *out);
+
 /* Copy the mask to host: h_blk_col [nrt*kkeep] int32, h_nm_bits [nrt*block_rows *
  * nblk*block_k/32] uint32.  Either may be NULL.  Synchronises `stream`. */
 CRISP_API crisp_status_t crisp_mask_export(crisp_mask_t mask, int32_t *h_blk_col, uint32_t *h_nm_bits,

@@ -60,6 +60,7 @@ def load(path: Optional[str] = None):
         "crisp_keep_count": [P(LayerDesc), P(i32), P(i32)],
         "crisp_mask_sizes": [P(LayerDesc), P(sz), P(sz)],
         "crisp_build_mask": [vp, i64, P(LayerDesc), vp, vp, vp, P(vp)],
+        "crisp_build_mask_static": [vp, i64, P(LayerDesc), vp, vp, P(vp)],
         "crisp_mask_export": [vp, vp, vp, vp],
         "crisp_mask_info": [vp, P(LayerDesc), P(i32), P(i32), P(i32)],
         "crisp_encode_sizes": [vp, P(sz), P(sz)],
@@ -140,6 +141,20 @@ def crisp_build_mask(d_saliency, ld_s: int, desc: LayerDesc, d_mask_buf, d_works
     out = C.c_void_p()
     _check(load().crisp_build_mask(_ptr(d_saliency), ld_s, C.byref(desc), _ptr(d_mask_buf), _ptr(d_workspace),
                                    _stream(stream), C.byref(out)), "crisp_build_mask")
+    return out.value
+
+
+STATIC_SCRATCH_BYTES = 256 * 1024
+
+
+def crisp_build_mask_static(d_saliency, ld_s: int, desc: LayerDesc, d_mask_buf, stream=None) -> int:
+    """crisp_build_mask without a caller-provided workspace: the scratch is a fixed array inside
+    the library, for callers that may not allocate device memory.  Layers whose workspace exceeds
+    STATIC_SCRATCH_BYTES raise CrispError(BUFFER_TOO_SMALL).  Calls share that array, so they must
+    not overlap on the GPU."""
+    out = C.c_void_p()
+    _check(load().crisp_build_mask_static(_ptr(d_saliency), ld_s, C.byref(desc), _ptr(d_mask_buf),
+                                          _stream(stream), C.byref(out)), "crisp_build_mask_static")
     return out.value
 
 
