@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".{os.getpid()}.tmp"
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-        ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources() + ["-lcuda"]
+        ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

@@ -1,5 +1,6 @@
 // C ABI of libcrisp: argument checking, buffer carving and kernel dispatch.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -41,6 +42,21 @@ crisp_status_t make_geometry(const crisp_layer_desc_t *d, Geometry *g) {
 void fill_desc(const Geometry &g, double keep_ratio, crisp_layer_desc_t *d) {
     d->rows = g.rows; d->k = g.k; d->n = g.n; d->m = g.m;
     d->block_rows = g.bm; d->block_k = g.bk; d->keep_ratio = keep_ratio; d->score_mode = g.score_mode;
+}
+
+// Which execution image crisp_encode lays out.  Default: the 2:4 sparse-MMA image when every aligned
+// 4-group keeps at most two values (n <= 2), the zero-expanded dense-tile image otherwise.  The
+// environment variable CRISP_EXEC_IMAGE = dense | none overrides it (for measurements).
+int image_kind(const Geometry &g) {
+    const char *e = std::getenv("CRISP_EXEC_IMAGE");
+    if (e && !std::strcmp(e, "none")) return CRISP_PATH_DIRECT;
+    if (e && !std::strcmp(e, "dense")) return CRISP_PATH_DENSE;
+    return crisp::tc_pattern_is_sparse(g) ? CRISP_PATH_SPARSE : CRISP_PATH_DENSE;
+}
+
+size_t exec_payload_bytes(const Geometry &g, int kind) {
+    if (kind == CRISP_PATH_DIRECT) return 0;
+    return crisp::tc_image_layout(g, kind == CRISP_PATH_SPARSE).total_bytes;
 }
 
 size_t blk_col_bytes(const Geometry &g) { return align_up((size_t)g.nrt * g.kkeep * sizeof(int32_t) + 4); }
@@ -133,7 +149,7 @@ crisp_status_t crisp_encode_sizes(crisp_mask_t mask, size_t *canonical_bytes, si
     if (!mask) return CRISP_INVALID_ARG;
     const Geometry &g = mask->g;
     if (canonical_bytes) *canonical_bytes = blk_col_bytes(g) + vals_bytes(g) + idx_bytes(g);
-    if (exec_bytes) *exec_bytes = kAlign;   // status word only: no tensor-core image yet
+    if (exec_bytes) *exec_bytes = kAlign + exec_payload_bytes(g, image_kind(g));
     return CRISP_OK;
 }
 
@@ -155,14 +171,17 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     h->d_idx = reinterpret_cast<uint32_t *>(p);
     h->d_status = reinterpret_cast<int32_t *>(d_exec_buf);
     h->d_exec = reinterpret_cast<uint8_t *>(d_exec_buf) + kAlign;
-    h->exec_payload_bytes = 0;
-    h->exec_kind = CRISP_PATH_DIRECT;
+    h->exec_kind = image_kind(g);
+    h->exec_payload_bytes = exec_payload_bytes(g, h->exec_kind);
     h->forced_path = -1;
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
     if (e == cudaSuccess)
         e = crisp::launch_encode_canonical(d_w_bf16, ld_w, g, mask->d_blk_col, mask->d_nm_bits,
                                            h->d_blk_col, h->d_vals, h->d_idx, st);
+    if (e == cudaSuccess && h->exec_kind != CRISP_PATH_DIRECT)
+        e = crisp::launch_build_image(g, h->exec_kind == CRISP_PATH_SPARSE, h->d_blk_col, h->d_vals, h->d_idx,
+                                      h->d_exec, st);
     if (e != cudaSuccess) { delete h; return CRISP_CUDA_ERROR; }
     *out = h;
     return CRISP_OK;
@@ -214,8 +233,17 @@ crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ld
     if (ncols <= 0 || ldx < ncols || ldy < ncols) return CRISP_BAD_SHAPE;
     if (!aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype ? 4 : 2)) return CRISP_INVALID_ARG;
     if ((ncols + 63) / 64 > 0x7FFFFFFFll) return CRISP_UNSUPPORTED;
-    cudaError_t e = crisp::launch_spmm_direct(h->g, h->d_blk_col, h->d_vals, h->d_idx, d_x_bf16, ldx, ncols,
-                                              d_y, ldy, y_dtype, (cudaStream_t)stream);
+    int path = h->forced_path >= 0 ? h->forced_path : h->exec_kind;
+    if (h->g.kkeep == 0 || !crisp::tc_operands_ok(d_x_bf16, ldx, d_y, ldy, y_dtype, ncols)) path = CRISP_PATH_DIRECT;
+    cudaError_t e;
+    if (path == CRISP_PATH_DIRECT) {
+        e = crisp::launch_spmm_direct(h->g, h->d_blk_col, h->d_vals, h->d_idx, d_x_bf16, ldx, ncols,
+                                      d_y, ldy, y_dtype, (cudaStream_t)stream);
+    } else {
+        const char *nt = std::getenv("CRISP_TC_NT");     // column boxes per CTA tile, tuning only
+        e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx, ncols,
+                                  d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, (cudaStream_t)stream);
+    }
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }
 

@@ -66,6 +66,24 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
 cudaError_t launch_decode(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                           const uint32_t *d_idx, uint16_t *d_w, int64_t ld, cudaStream_t st);
 
+// spmm_tc.cu: tensor-core path and its execution image
+struct TcImageLayout {
+    int r;                  // row tiles per 128-row CTA tile
+    int nst;                // 128-row CTA tiles
+    int wcap;               // capacity of one CTA tile's walk list (union of its row tiles' kept blocks)
+    uint32_t a_bytes;       // weight tile bytes per walk entry
+    uint32_t entry_bytes;   // weight tile + metadata
+    size_t walk_col_off, walk_len_off, image_off, total_bytes;   // offsets inside the exec payload
+};
+bool tc_pattern_is_sparse(const Geometry &g);
+TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
+cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
+                               const uint32_t *d_idx, uint8_t *d_exec, cudaStream_t st);
+bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols);
+cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
+                           const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
+                           int nt_override, cudaStream_t st);
+
 // spmm_direct.cu
 cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, const uint16_t *d_x, int64_t ldx, int64_t ncols,

@@ -1,0 +1,627 @@
+// Tensor-core SpMM over kept blocks (sm_100a): TMA-staged, warp-specialised, tcgen05 MMA with
+// TMEM accumulators.  Sec. III-E of the paper, mapped onto B200:
+//   step 1 (load the activations of kept blocks): the producer warp walks the kept-block list of
+//           a 128-row tile and issues, per kept block, one bulk copy of the weight tile (from the
+//           execution image) and TMA tensor loads of the X rows [blk_col*Bk, +Bk) only;
+//   step 2 (select activations by offset): either the 2:4 metadata drives tcgen05.mma.sp's operand
+//           selection (sparse image), or the weight tile is stored zero-expanded so that the
+//           selection is the identity (dense image);
+//   step 3 (multiply-accumulate): tcgen05.mma, fp32 accumulators in tensor memory, epilogue warps
+//           convert and TMA-store Y.
+// A CTA is persistent over (128-row tile, column tile) pairs; all row tiles of a layer have the same
+// number of kept blocks (uniform block pruning, Sec. III-A), so tiles are load-balanced by construction.
+//
+// The execution image is built by the kernels at the bottom of this file from the canonical format.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "crisp_internal.h"
+
+namespace crisp {
+
+namespace {
+
+constexpr int kTileM = 128;                 // rows per CTA tile = MMA M
+constexpr int kBoxN = 64;                   // columns per TMA box of X (128 bytes, one swizzle span)
+constexpr int kThreads = 192;               // warp 0 producer, warp 1 MMA issuer, warps 2..5 epilogue
+constexpr int kEpiWarps = 4;
+constexpr uint32_t kStageTileBytes = 4096;  // one epilogue staging tile: 32 rows x 128 bytes
+constexpr uint32_t kMetaBytes = 2048;       // 128 rows x 16 bytes of 2:4 metadata per kept block
+constexpr uint32_t kSmemBudget = 232448 - 1024;
+constexpr unsigned long long kWaitLimitCycles = 4000000000ull;   // ~2 s: then report CRISP_TIMEOUT
+
+struct TcParams {
+    const uint8_t *image;       // per walk entry: weight tile (+ metadata), entry_bytes each
+    const int32_t *walk_col;    // [nst, wcap] block column of each walk entry
+    const int32_t *walk_len;    // [nst]
+    int32_t *status;
+    void *y;                    // for edge chunks that TMA cannot clip exactly
+    int64_t ldy;
+    int nst, wcap, bk, n_col_tiles, num_tiles, rows;
+    int64_t ncols;
+    uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait: gives up after kWaitLimitCycles or when another role has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > kWaitLimitCycles) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_dense(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_sparse(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t acc, uint32_t meta_tmem) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%5], %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc), "r"(meta_tmem) : "memory");
+}
+__device__ __forceinline__ void tmem_copy_128x128b(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (Blackwell format, version 1).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
+}
+constexpr uint32_t kLayoutNone = 0, kLayoutSw128 = 2;
+
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B MN-major (X has ncols contiguous), M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool sparse) {
+    return (sparse ? (1u << 2) : 0u) | (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// ----------------------------------------------------------------------------------- kernel
+//
+// Shared memory (1024-byte aligned): num_stages x [weight tile | metadata (sparse) | NT boxes of X]
+//                                    | 4 warps x 2 staging tiles | barriers | TMEM base | abort flag
+// Weight tile layout (no swizzle, K-major): [k/8][row][8 elements], i.e. 8x16-byte core matrices are
+// contiguous, 128 bytes between 8-row groups, 2048 bytes between 16-byte K chunks.
+// X box layout: TMA SWIZZLE_128B, 64 columns (128 bytes) x bk rows; MN-major operand with 1024 bytes
+// between 8-row K groups and box_bytes between 64-column groups.
+template <int NT, bool kSparse, int kAccStages, typename OutT>
+__global__ void __launch_bounds__(kThreads, 1)
+spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, TcParams p) {
+    constexpr int kTileN = NT * kBoxN;
+    constexpr int kMetaCols = kSparse ? 8 : 0;                       // two 4-column metadata buffers
+    constexpr int kTmemCols = (kAccStages * kTileN + kMetaCols) <= 256 ? 256 : 512;
+    static_assert(kAccStages * kTileN + kMetaCols <= 512, "tensor memory is 512 columns");
+    constexpr int kOutCols = 128 / (int)sizeof(OutT);                // columns of one 128-byte staging row
+    constexpr uint32_t kIdesc = make_idesc(kTileN, kSparse);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t ring = smem_base;
+    const uint32_t staging = ring + p.num_stages * p.stage_bytes;
+    const uint32_t ctrl = staging + kEpiWarps * 2 * kStageTileBytes;
+    uint8_t *ctrl_gen = smem_gen + (ctrl - smem_base);
+    // barriers: full[s], empty[s] (s < 8), tmem_full[2], tmem_empty[2]
+    const uint32_t bar_full = ctrl, bar_empty = ctrl + 64, bar_tfull = ctrl + 128, bar_tempty = ctrl + 144;
+    volatile uint32_t *tmem_base_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 160);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + 164);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < p.num_stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_base_slot)), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+    const uint32_t tx_bytes = p.entry_bytes + NT * p.box_bytes;
+
+    if (warp == 0) {
+        // ------------------------------------------------ producer: step 1, kept blocks only
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                const int st = t % p.nst, ct = t / p.nst;
+                const int len = p.walk_len[st];
+                const int32_t *cols = p.walk_col + (int64_t)st * p.wcap;
+                const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
+                for (int e = 0; e < len; ++e) {
+                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) break;
+                    const uint32_t dst = ring + s * p.stage_bytes;
+                    mbar_expect_tx(bar_full + 8 * s, tx_bytes);
+                    bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, bar_full + 8 * s);
+                    const int krow = cols[e] * p.bk;
+#pragma unroll
+                    for (int b = 0; b < NT; ++b)
+                        tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow,
+                                    bar_full + 8 * s);
+                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer: steps 2 + 3
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
+            for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                const int len = p.walk_len[t % p.nst];
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1u, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kTileN;
+                bool ok = true;
+                for (int e = 0; e < len; ++e) {
+                    if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_smem = ring + s * p.stage_bytes;
+                    const uint32_t x_smem = a_smem + p.entry_bytes;
+                    if constexpr (kSparse) {
+                        const uint32_t meta_tmem = tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                        tmem_copy_128x128b(meta_tmem, make_smem_desc(a_smem + p.a_bytes, 128, 128, kLayoutNone));
+                        for (int j = 0; j < p.bk / 32; ++j) {
+                            const uint64_t ad = make_smem_desc(a_smem + j * 4096, 2048, 128, kLayoutNone);
+                            const uint64_t bd = make_smem_desc(x_smem + j * 4096, p.box_bytes, 1024, kLayoutSw128);
+                            mma_sparse(d_tmem, ad, bd, kIdesc | (uint32_t)(j & 1), (e | j) ? 1u : 0u, meta_tmem + (j & ~1));
+                        }
+                        meta_buf ^= 1u;
+                    } else {
+                        for (int j = 0; j < p.bk / 16; ++j) {
+                            const uint64_t ad = make_smem_desc(a_smem + j * 4096, 2048, 128, kLayoutNone);
+                            const uint64_t bd = make_smem_desc(x_smem + j * 2048, p.box_bytes, 1024, kLayoutSw128);
+                            mma_dense(d_tmem, ad, bd, kIdesc, (e | j) ? 1u : 0u);
+                        }
+                    }
+                    mma_commit(bar_empty + 8 * s);          // stage reusable once these MMAs have read it
+                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                mma_commit(bar_tfull + 8 * acc);            // accumulator complete
+                if (++acc == kAccStages) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue: TMEM -> registers -> smem -> TMA store
+        const int q = warp & 3;                             // TMEM lane quarter this warp may access
+        const uint32_t stg = staging + (uint32_t)(warp - 2) * 2 * kStageTileBytes;
+        uint8_t *stg_gen = smem_gen + (stg - smem_base);
+        uint32_t acc = 0, acc_ph = 0, buf = 0;
+        for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
+            const int st = t % p.nst, ct = t / p.nst;
+            int go = 0;                                      // lane 0 waits, the warp follows it
+            if (lane == 0) go = !*abort_flag && mbar_wait(bar_tfull + 8 * acc, acc_ph, abort_flag);
+            go = __shfl_sync(0xFFFFFFFFu, go, 0);
+            if (!go) break;
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
+#pragma unroll 1
+            for (int c = 0; c < kTileN / kOutCols; ++c) {
+                uint32_t out[32];                            // one 128-byte row per lane
+                if constexpr (sizeof(OutT) == 2) {
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32(t_addr + c * 64, r0);
+                    tmem_ld32(t_addr + c * 64 + 32, r1);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        out[i] = pack_bf16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+                        out[16 + i] = pack_bf16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
+                    }
+                } else {
+                    tmem_ld32(t_addr + c * 32, out);
+                    tmem_ld_wait();
+                }
+                const int x0 = ct * kTileN + c * kOutCols, y0 = st * kTileM + 32 * q;
+                // TMA clips a store at 16-byte granularity: a chunk that crosses an ncols whose byte
+                // offset is not a multiple of 16 is written with guarded plain stores instead
+                if (x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
+                    const int row = y0 + lane;
+                    if (row < p.rows && x0 < p.ncols) {
+                        OutT *dst = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy + x0;
+                        const int nvalid = (int)(p.ncols - x0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            if constexpr (sizeof(OutT) == 2) {
+                                if (2 * i < nvalid) dst[2 * i] = (OutT)(out[i] & 0xFFFFu);
+                                if (2 * i + 1 < nvalid) dst[2 * i + 1] = (OutT)(out[i] >> 16);
+                            } else {
+                                if (i < nvalid) dst[i] = __uint_as_float(out[i]);
+                            }
+                        }
+                    }
+                    continue;
+                }
+                if (lane == 0) bulk_wait_read<1>();          // the staging tile written two stores ago is free
+                __syncwarp();
+                uint8_t *tile = stg_gen + buf * kStageTileBytes + lane * 128;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)                  // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
+                    *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
+                        make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (x0 < p.ncols && y0 < p.rows) tma_store_2d(&map_y, stg + buf * kStageTileBytes, x0, y0);
+                    bulk_commit();
+                }
+                buf ^= 1u;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            if (++acc == kAccStages) { acc = 0; acc_ph ^= 1u; }
+        }
+        if (lane == 0) bulk_wait_read<0>();
+    }
+
+    // ------------------------------------------------ teardown (every wait above is bounded)
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)CRISP_TIMEOUT);
+        // let copies that may still be in flight land before shared memory is released
+        const unsigned long long t0 = clock64();
+        while ((unsigned long long)(clock64() - t0) < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// --------------------------------------------------------------------- execution image kernels
+
+// Union walk of the r = 128 / bm row tiles that share one CTA tile: ascending block columns.
+__global__ void build_walk_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int wcap,
+                                  int32_t *__restrict__ walk_col, int32_t *__restrict__ walk_len) {
+    const int st = blockIdx.x * blockDim.x + threadIdx.x;
+    const int nst = (g.nrt + r - 1) / r;
+    if (st >= nst) return;
+    int pos[4] = {0, 0, 0, 0};
+    int len = 0;
+    for (;;) {
+        int best = 0x7FFFFFFF;
+        for (int i = 0; i < r; ++i) {
+            const int rt = st * r + i;
+            if (rt < g.nrt && pos[i] < g.kkeep) best = min(best, blk_col[(int64_t)rt * g.kkeep + pos[i]]);
+        }
+        if (best == 0x7FFFFFFF) break;
+        for (int i = 0; i < r; ++i) {
+            const int rt = st * r + i;
+            if (rt < g.nrt && pos[i] < g.kkeep && blk_col[(int64_t)rt * g.kkeep + pos[i]] == best) ++pos[i];
+        }
+        walk_col[(int64_t)st * wcap + len++] = best;
+    }
+    walk_len[st] = len;
+}
+
+// One CTA per kept block: scatter its values into the (pre-zeroed) tile of its walk entry.
+// Dense image: element (row, k) of the tile at [k/8][row][k%8].
+// Sparse image: per 4-group two slots (ascending position, zero-padded), slot pair p = k/4 stored at
+// compressed column 2p + slot, same [c/8][row][c%8] layout; metadata word j = k/32 of row L' holds
+// 16 bits for row (16*(row/16) + row%8) and 16 bits for that row + 8, where
+// L' = row%8 + 8*((k/16)%2) + 16*(row/16); nibble g%4... of a 4-group = idx0 | idx1 << 2.
+template <bool kSparse>
+__global__ void __launch_bounds__(256)
+build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16_t *__restrict__ vals,
+                   const uint32_t *__restrict__ idx, int r, int wcap, const int32_t *__restrict__ walk_col,
+                   const int32_t *__restrict__ walk_len, uint32_t a_bytes, uint32_t entry_bytes,
+                   uint8_t *__restrict__ image) {
+    const int blk = blockIdx.x;
+    const int rt = blk / g.kkeep;
+    const int jb = blk_col[blk];
+    const int st = rt / r;
+    __shared__ int s_entry;
+    if (threadIdx.x == 0) {
+        int lo = 0, hi = walk_len[st] - 1, found = 0;
+        const int32_t *wc = walk_col + (int64_t)st * wcap;
+        while (lo <= hi) {
+            const int mid = (lo + hi) >> 1;
+            if (wc[mid] == jb) { found = mid; break; }
+            if (wc[mid] < jb) lo = mid + 1; else hi = mid - 1;
+        }
+        s_entry = found;
+    }
+    __syncthreads();
+    uint8_t *tile = image + ((int64_t)st * wcap + s_entry) * entry_bytes;
+    const int row0 = (rt % r) * g.bm;
+    const int groups = g.groups();
+    const int64_t vpb = g.vals_per_block();
+    const uint16_t *vb = vals + (int64_t)blk * vpb;
+    const uint32_t *ib = idx + (int64_t)blk * (vpb * g.idx_bits / 32);
+    const uint32_t field = (1u << g.idx_bits) - 1u;
+    if constexpr (!kSparse) {
+        for (int o = threadIdx.x; o < (int)vpb; o += blockDim.x) {
+            const int item = o / g.n;
+            const int lr = item / groups, gi = item - lr * groups;
+            const int bit = o * g.idx_bits;
+            uint32_t t = ib[bit >> 5] >> (bit & 31);
+            if ((bit & 31) + g.idx_bits > 32) t |= ib[(bit >> 5) + 1] << (32 - (bit & 31));
+            t &= field;
+            const int k = gi * g.m + (int)t, row = row0 + lr;
+            *reinterpret_cast<uint16_t *>(tile + (k >> 3) * 2048 + row * 16 + (k & 7) * 2) = vb[o];
+        }
+    } else {
+        // one thread per (local row, 4-group): at most two kept values by construction
+        const int quads = g.bk / 4;
+        uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
+        for (int item = threadIdx.x; item < g.bm * quads; item += blockDim.x) {
+            const int lr = item / quads, qd = item - lr * quads;
+            const int row = row0 + lr;
+            // kept values of this row whose position falls into [4*qd, 4*qd+4)
+            const int gi = (qd * 4) / g.m;
+            uint16_t v[2] = {0, 0};
+            int pos[2] = {0, 0}, cnt = 0;
+            for (int vv = 0; vv < g.n; ++vv) {
+                const int o = (lr * groups + gi) * g.n + vv;
+                const int bit = o * g.idx_bits;
+                uint32_t t = ib[bit >> 5] >> (bit & 31);
+                if ((bit & 31) + g.idx_bits > 32) t |= ib[(bit >> 5) + 1] << (32 - (bit & 31));
+                t &= field;
+                const int k = gi * g.m + (int)t;
+                if ((k >> 2) == qd && cnt < 2) { v[cnt] = vb[o]; pos[cnt] = k & 3; ++cnt; }
+            }
+            if (cnt == 0) { pos[0] = 0; pos[1] = 1; }
+            else if (cnt == 1) {
+                if (pos[0] == 3) { v[1] = v[0]; v[0] = 0; pos[1] = 3; pos[0] = 0; }
+                else pos[1] = 3;
+            }
+            const int c0 = 2 * qd;
+            *reinterpret_cast<uint16_t *>(tile + (c0 >> 3) * 2048 + row * 16 + (c0 & 7) * 2) = v[0];
+            *reinterpret_cast<uint16_t *>(tile + ((c0 + 1) >> 3) * 2048 + row * 16 + ((c0 + 1) & 7) * 2) = v[1];
+            const uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
+            const int k0 = qd * 4;
+            const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
+            const int word = k0 >> 5;
+            const int shift = (k0 & 15) + 16 * ((row >> 3) & 1);
+            atomicOr(&meta[lrow * 4 + word], nib << shift);
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, uint64_t inner,
+                 uint64_t outer, uint64_t ld_elems, uint32_t box_inner, uint32_t box_outer) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {ld_elems * (uint64_t)elem_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NT, bool kSparse, int kAccStages, typename OutT>
+cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const TcParams &p, int grid, size_t smem,
+                           cudaStream_t st) {
+    auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT>;
+    static size_t configured = 0;                       // largest dynamic shared memory opted into so far
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = smem;
+    }
+    kern<<<grid, kThreads, smem, st>>>(mx, my, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ interface to crisp_api.cu
+
+bool tc_pattern_is_sparse(const Geometry &g) { return g.n <= 2; }   // <= 2 kept per aligned 4-group
+
+TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
+    TcImageLayout L;
+    L.r = kTileM / g.bm;
+    L.nst = (g.nrt + L.r - 1) / L.r;
+    const int64_t cap = (int64_t)L.r * g.kkeep;
+    L.wcap = (int)(cap < g.nblk ? cap : g.nblk);
+    L.a_bytes = (uint32_t)(kTileM * g.bk * 2) / (sparse ? 2 : 1);
+    L.entry_bytes = L.a_bytes + (sparse ? kMetaBytes : 0);
+    L.walk_col_off = 0;
+    L.walk_len_off = align_up((size_t)L.nst * L.wcap * sizeof(int32_t) + 4);
+    L.image_off = L.walk_len_off + align_up((size_t)L.nst * sizeof(int32_t) + 4);
+    L.total_bytes = L.image_off + align_up((size_t)L.nst * L.wcap * L.entry_bytes + 16);
+    return L;
+}
+
+cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
+                               const uint32_t *d_idx, uint8_t *d_exec, cudaStream_t st) {
+    const TcImageLayout L = tc_image_layout(g, sparse);
+    if (g.nrt * g.kkeep == 0) return cudaSuccess;
+    int32_t *walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
+    int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
+    uint8_t *image = d_exec + L.image_off;
+    cudaError_t e = cudaMemsetAsync(image, 0, (size_t)L.nst * L.wcap * L.entry_bytes, st);
+    if (e != cudaSuccess) return e;
+    build_walk_kernel<<<(L.nst + 127) / 128, 128, 0, st>>>(g, d_blk_col, L.r, L.wcap, walk_col, walk_len);
+    if (sparse)
+        build_image_kernel<true><<<g.nrt * g.kkeep, 256, 0, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
+                                                                   walk_len, L.a_bytes, L.entry_bytes, image);
+    else
+        build_image_kernel<false><<<g.nrt * g.kkeep, 256, 0, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
+                                                                    walk_len, L.a_bytes, L.entry_bytes, image);
+    return cudaGetLastError();
+}
+
+// Whether the tensor-core kernel can address these operands (TMA: 16-byte aligned base and pitch).
+bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols) {
+    const int ye = y_dtype ? 4 : 2;
+    return (reinterpret_cast<uintptr_t>(x) % 16 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0) &&
+           (ldx * 2) % 16 == 0 && (ldy * ye) % 16 == 0 && ncols < (1ll << 31) && encode_tiled_fn() != nullptr;
+}
+
+cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
+                           const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
+                           int nt_override, cudaStream_t st) {
+    const TcImageLayout L = tc_image_layout(g, sparse);
+    static int sm_count = 0;
+    if (!sm_count) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (sm_count <= 0) sm_count = 148;
+    }
+    // column tile: 4 boxes (256 columns) when two accumulators fit beside the metadata, else 3
+    int nt = (nt_override >= 1 && nt_override <= 4) ? nt_override : (sparse ? 3 : 4);
+    const int64_t boxes = (ncols + kBoxN - 1) / kBoxN;
+    if (boxes < nt) nt = (int)boxes;
+    TcParams p;
+    p.image = d_exec + L.image_off;
+    p.walk_col = reinterpret_cast<const int32_t *>(d_exec + L.walk_col_off);
+    p.walk_len = reinterpret_cast<const int32_t *>(d_exec + L.walk_len_off);
+    p.status = d_status;
+    p.nst = L.nst; p.wcap = L.wcap; p.bk = g.bk; p.rows = g.rows; p.ncols = ncols; p.y = d_y; p.ldy = ldy;
+    p.n_col_tiles = (int)((ncols + nt * kBoxN - 1) / (nt * kBoxN));
+    const int64_t tiles = (int64_t)p.n_col_tiles * L.nst;
+    if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    p.num_tiles = (int)tiles;
+    p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes;
+    p.box_bytes = (uint32_t)(kBoxN * g.bk * 2);
+    p.stage_bytes = p.entry_bytes + nt * p.box_bytes;
+    const uint32_t fixed = kEpiWarps * 2 * kStageTileBytes + 256;
+    uint32_t stages = (kSmemBudget - fixed) / p.stage_bytes;
+    if (stages > 8) stages = 8;
+    if (stages < 2) return cudaErrorInvalidValue;
+    p.num_stages = stages;
+    const size_t smem = (size_t)stages * p.stage_bytes + fixed + 1024;
+
+    CUtensorMap mx, my;
+    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, (uint64_t)ncols, (uint64_t)g.k, (uint64_t)ldx,
+                     kBoxN, (uint32_t)g.bk))
+        return cudaErrorInvalidValue;
+    const bool f32 = y_dtype != 0;
+    if (!make_map_2d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, f32 ? 4 : 2, d_y,
+                     (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, 32))
+        return cudaErrorInvalidValue;
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+
+#define CRISP_TC_LAUNCH(NTV, SP, ACC)                                                                     \
+    (f32 ? launch_variant<NTV, SP, ACC, float>(mx, my, p, grid, smem, st)                                 \
+         : launch_variant<NTV, SP, ACC, uint16_t>(mx, my, p, grid, smem, st))
+    if (sparse) {
+        switch (nt) {
+            case 1: return CRISP_TC_LAUNCH(1, true, 2);
+            case 2: return CRISP_TC_LAUNCH(2, true, 2);
+            case 3: return CRISP_TC_LAUNCH(3, true, 2);
+            default: return CRISP_TC_LAUNCH(4, true, 1);
+        }
+    }
+    switch (nt) {
+        case 1: return CRISP_TC_LAUNCH(1, false, 2);
+        case 2: return CRISP_TC_LAUNCH(2, false, 2);
+        case 3: return CRISP_TC_LAUNCH(3, false, 2);
+        default: return CRISP_TC_LAUNCH(4, false, 2);
+    }
+#undef CRISP_TC_LAUNCH
+}
+
+}  // namespace crisp

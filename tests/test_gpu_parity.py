@@ -48,9 +48,31 @@ CASES = [
 ]
 
 
+# which execution image crisp_encode lays out: the default choice (2:4 sparse MMA when n <= 2, dense
+# tiles otherwise), dense tiles forced, or none (CUDA-core kernel on the canonical format)
+IMAGES = ["auto", "dense", "none"]
+
+
+@pytest.fixture(params=IMAGES)
+def image(request, monkeypatch):
+    if request.param == "auto":
+        monkeypatch.delenv("CRISP_EXEC_IMAGE", raising=False)
+    else:
+        monkeypatch.setenv("CRISP_EXEC_IMAGE", request.param)
+    return request.param
+
+
+def expected_path(B, image, n, kkeep=1):
+    if image == "none":
+        return B.PATH_DIRECT
+    if image == "dense":
+        return B.PATH_DENSE
+    return B.PATH_SPARSE if n <= 2 else B.PATH_DENSE
+
+
 @pytest.mark.parametrize("rows,k,ncols,n,m,bm,bk,keep", CASES)
 @pytest.mark.parametrize("y_dtype", [0, 1])
-def test_layer_matches_oracle(env, rows, k, ncols, n, m, bm, bk, keep, y_dtype):
+def test_layer_matches_oracle(env, image, rows, k, ncols, n, m, bm, bk, keep, y_dtype):
     B, torch = env
     w, s, x = rand_inputs(rows, k, ncols, seed=rows + k + ncols)
     mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
@@ -58,10 +80,17 @@ def test_layer_matches_oracle(env, rows, k, ncols, n, m, bm, bk, keep, y_dtype):
     assert_mask_and_encoding_equal(L, mk, vals, idx)
     dec = L.decode().view(torch.int16).cpu().numpy().view(np.uint16)
     assert np.array_equal(dec, wb)
-    y = L.spmm(bf16_dev(x, torch), y_dtype=y_dtype)
+    # ncols padded to a multiple of 8 in memory so that the tensor-core kernels can address X and Y
+    ld = (ncols + 7) // 8 * 8
+    xbuf = torch.zeros((k, ld), dtype=torch.bfloat16, device="cuda")
+    xbuf[:, :ncols] = bf16_dev(x, torch)
+    ybuf = torch.full((rows, ld), 5.0, dtype=torch.float32 if y_dtype else torch.bfloat16, device="cuda")
+    assert L.bytes_model(ncols, y_dtype)["path"] == expected_path(B, image, n)
+    L.spmm(xbuf[:, :ncols], y=ybuf[:, :ncols], y_dtype=y_dtype)
     torch.cuda.synchronize()
     assert L.device_status() == 0
-    check_tolerance(y_to_f64(y, torch), oracle.spmm_fp64(wd, x))
+    check_tolerance(y_to_f64(ybuf[:, :ncols], torch), oracle.spmm_fp64(wd, x))
+    assert torch.all(ybuf[:, ncols:] == 5.0)                             # nothing written past ncols
     L.close()
 
 
@@ -137,7 +166,7 @@ def test_no_kept_block_writes_zeros(env):
 
 
 @pytest.mark.parametrize("n,m,bm,bk,keep", [(2, 4, 32, 64, 0.5), (1, 8, 64, 32, 0.25), (4, 8, 128, 64, 1.0)])
-def test_identity_activation_is_bit_exact(env, n, m, bm, bk, keep):
+def test_identity_activation_is_bit_exact(env, image, n, m, bm, bk, keep):
     """X = I: every output is a single product by 1, exact in fp32 and in bf16, so Y must equal
     the decoded weight bit for bit; this pins every index and offset path."""
     B, torch = env
@@ -153,7 +182,7 @@ def test_identity_activation_is_bit_exact(env, n, m, bm, bk, keep):
     assert np.array_equal(y_to_f64(y, torch), oracle.spmm_fp64(wd, wl.f32_to_bf16_bits(np.eye(k, dtype=np.float32))))
 
 
-def test_config1_full(env):
+def test_config1_full(env, image):
     B, torch = env
     l = wl.config1()[0]
     w, s, x = wl.make_layer_inputs(l)
@@ -164,7 +193,7 @@ def test_config1_full(env):
     check_tolerance(y_to_f64(y, torch), oracle.spmm_fp64(wd, x))
 
 
-def test_config2_full(env):
+def test_config2_full(env, image):
     B, torch = env
     l = wl.config2()[0]
     w, s, x = wl.make_layer_inputs(l)
