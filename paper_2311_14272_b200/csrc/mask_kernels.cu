@@ -26,6 +26,20 @@ __device__ __forceinline__ uint32_t canonical_key(float s) {
     return u;
 }
 
+// Raw bits of eight consecutive saliency values; the caller guarantees row < rows, k0 + 8 <= k and
+// 16-byte alignment.  Kept free of branches so that several of these can be in flight per lane.
+__device__ __forceinline__ void load8_raw(const float *__restrict__ s, int64_t ld, int64_t row, int64_t k0,
+                                          uint32_t key[8]) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(s + row * ld + k0);
+    const uint4 a = __ldg(p), b = __ldg(p + 1);
+    key[0] = a.x; key[1] = a.y; key[2] = a.z; key[3] = a.w;
+    key[4] = b.x; key[5] = b.y; key[6] = b.z; key[7] = b.w;
+}
+__device__ __forceinline__ uint32_t canonical_bits(uint32_t u) {
+    u &= 0x7FFFFFFFu;
+    return u > 0x7F800000u ? 0u : min(u, 0x7F7FFFFFu);
+}
+
 // Eight consecutive saliency values of one row, zero beyond the matrix.
 __device__ __forceinline__ void load8(const float *__restrict__ s, int64_t ld, int rows, int k,
                                       int64_t row, int64_t k0, bool vec_ok, uint32_t key[8]) {
@@ -48,29 +62,61 @@ __device__ __forceinline__ void load8(const float *__restrict__ s, int64_t ld, i
     }
 }
 
+// K-M0.  One warp per (row, 1024-element segment): eight 16-byte loads per lane are issued before
+// any is used, partial maxima are combined per warp and per CTA, one atomic per CTA.
 __global__ void __launch_bounds__(256)
 max_key_kernel(const float *__restrict__ s, int64_t ld, int rows, int k, bool vec_ok,
                uint32_t *__restrict__ max_key) {
-    const int chunks = (k + 7) / 8;
-    const int64_t total = (int64_t)rows * chunks;
+    __shared__ uint32_t s_best[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int segs = (k + 1023) / 1024;
+    const int64_t items = (int64_t)rows * segs;
+    const int64_t nwarps = (int64_t)gridDim.x * 8;
     uint32_t best = 0u;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = i / chunks;
-        const int64_t k0 = (i - row * chunks) * 8;
-        uint32_t key[8];
-        load8(s, ld, rows, k, row, k0, vec_ok, key);
+    for (int64_t it = (int64_t)blockIdx.x * 8 + warp; it < items; it += nwarps) {
+        const int64_t row = it / segs;
+        const int64_t k0 = (it - row * segs) * 1024 + lane * 8;
+        uint32_t key[4][8];
+        if (vec_ok && (it - row * segs) * 1024 + 1024 <= k) {       // whole segment inside the row
 #pragma unroll
-        for (int j = 0; j < 8; ++j) best = max(best, key[j]);
+            for (int pass = 0; pass < 4; ++pass) load8_raw(s, ld, row, k0 + pass * 256, key[pass]);
+#pragma unroll
+            for (int pass = 0; pass < 4; ++pass)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) best = max(best, canonical_bits(key[pass][j]));
+        } else {
+#pragma unroll
+            for (int pass = 0; pass < 4; ++pass) load8(s, ld, rows, k, row, k0 + pass * 256, vec_ok, key[pass]);
+#pragma unroll
+            for (int pass = 0; pass < 4; ++pass)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) best = max(best, key[pass][j]);
+        }
     }
     best = __reduce_max_sync(0xFFFFFFFFu, best);
-    if ((threadIdx.x & 31) == 0 && best) atomicMax(max_key, best);
+    if (lane == 0) s_best[warp] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) best = max(best, s_best[w]);
+        if (best) atomicMax(max_key, best);
+    }
 }
 
 // Exponent of a positive finite float given by its bits (ilogb), denormals included.
 __device__ __forceinline__ int key_exponent(uint32_t key) {
     const int e = (int)(key >> 23);
     return e ? e - 127 : (31 - __clz(key)) - 149;
+}
+
+// floor(value * 2^(40 - e_max)) for a non-negative finite float given by its bits, in integer
+// arithmetic: the mantissa shifted by the exponent difference (exact, no rounding mode involved).
+__device__ __forceinline__ unsigned long long fixed_point_score(uint32_t key, int e_max) {
+    const int e = (int)(key >> 23);
+    const uint32_t mant = e ? ((key & 0x7FFFFFu) | 0x800000u) : key;           // value = mant * 2^(max(e,1) - 150)
+    const int sh = max(e, 1) - 150 + kScoreFractionBits - e_max;                 // <= 17 because value <= layer maximum
+    const uint32_t down = mant >> min(max(-sh, 0), 31);                          // mant < 2^24: shifts >= 24 give 0
+    const int up = max(sh, 0);                                                   // only one of the two shifts is non-zero
+    return ((unsigned long long)__funnelshift_l(down, 0u, up) << 32) | (unsigned long long)(down << up);
 }
 
 // Bit i of the result is set iff element i is among the N largest of its group of M
@@ -80,31 +126,40 @@ __device__ __forceinline__ uint32_t top_n_bits(const uint32_t key[8], int n) {
     uint32_t bits = 0u;
 #pragma unroll
     for (int g = 0; g < 8 / M; ++g) {
+        // rank[i] = number of elements that beat element i; for i < j, i beats j iff key[i] >= key[j]
+        int rank[M];
 #pragma unroll
-        for (int i = 0; i < M; ++i) {
-            int rank = 0;
+        for (int i = 0; i < M; ++i) rank[i] = 0;
 #pragma unroll
-            for (int j = 0; j < M; ++j) {
-                const uint32_t a = key[g * M + j], b = key[g * M + i];
-                rank += (a > b) || (a == b && j < i);
+        for (int i = 0; i < M; ++i)
+#pragma unroll
+            for (int j = i + 1; j < M; ++j) {
+                const int i_wins = key[g * M + i] >= key[g * M + j];
+                rank[j] += i_wins;
+                rank[i] += 1 - i_wins;
             }
-            bits |= (rank < n ? 1u : 0u) << (g * M + i);
-        }
+#pragma unroll
+        for (int i = 0; i < M; ++i) bits |= (rank[i] < n ? 1u : 0u) << (g * M + i);
     }
     return bits;
 }
 
-// One CTA covers bm rows x 256 k-elements.  Warp w takes rows w, w+8, ...; lane l owns the 8
-// elements at k = chunk*256 + 8*l of each of its rows, so every lane stays inside one block
-// column and keeps its partial block score in a register.
+constexpr int kM1Rows = 32;              // rows per CTA of K-M1 (divides every block height)
+constexpr int kM1RowsPerWarp = kM1Rows / (kM1Threads / 32);
+
+// K-M1.  One CTA covers 32 rows x 256 k-elements.  Warp w takes rows 4w..4w+3 (all loads issued
+// first); lane l owns the 8 elements at k = chunk*256 + 8*l of each row, so a lane stays inside one
+// block column and keeps its partial block score in a register.  Four lanes assemble one 32-bit
+// mask word and one partial score (a word never straddles a block: block_k is a multiple of 32).
 template <int M>
 __global__ void __launch_bounds__(kM1Threads)
 group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_ok,
                     const uint32_t *__restrict__ max_key, uint32_t *__restrict__ nm_bits,
                     unsigned long long *__restrict__ score) {
     __shared__ unsigned long long s_score[kM1ChunkK / 32 + 2];
-    const int rt = blockIdx.y;
-    const int chunk = blockIdx.x;
+    const int chunk = blockIdx.y;
+    const int64_t row0 = (int64_t)blockIdx.x * kM1Rows;
+    const int rt = (int)(row0 / g.bm);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t k0 = (int64_t)chunk * kM1ChunkK + lane * 8;
     const int first_blk = (chunk * kM1ChunkK) / g.bk;
@@ -112,26 +167,40 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
     __syncthreads();
 
     const uint32_t mk = *max_key;
-    const double scale = mk ? ldexp(1.0, kScoreFractionBits - key_exponent(mk)) : 0.0;
+    const int e_max = mk ? key_exponent(mk) : 0;
     const bool in_kp = k0 < g.kp();
-    unsigned long long acc = 0ull;
-    for (int r = warp; r < g.bm; r += kM1Threads / 32) {
-        const int64_t row = (int64_t)rt * g.bm + r;
-        uint32_t key[8];
-        load8(s, ld, g.rows, g.k, row, k0, vec_ok, key);
-        const uint32_t bits = top_n_bits<M>(key, g.n);
-        const uint32_t counted = g.score_mode == 0 ? bits : 0xFFu;
+    uint32_t key[kM1RowsPerWarp][8];
+    if (vec_ok && row0 + kM1Rows <= g.rows && (int64_t)(chunk + 1) * kM1ChunkK <= g.k) {   // interior tile
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if ((counted >> i) & 1u)
-                acc += __double2ull_rd((double)__uint_as_float(key[i]) * scale);
-        // four lanes assemble one 32-bit mask word
+        for (int i = 0; i < kM1RowsPerWarp; ++i) load8_raw(s, ld, row0 + warp * kM1RowsPerWarp + i, k0, key[i]);
+#pragma unroll
+        for (int i = 0; i < kM1RowsPerWarp; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) key[i][j] = canonical_bits(key[i][j]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < kM1RowsPerWarp; ++i)
+            load8(s, ld, g.rows, g.k, row0 + warp * kM1RowsPerWarp + i, k0, vec_ok, key[i]);
+    }
+    unsigned long long acc = 0ull;
+#pragma unroll
+    for (int i = 0; i < kM1RowsPerWarp; ++i) {
+        const int64_t row = row0 + warp * kM1RowsPerWarp + i;
+        const uint32_t bits = top_n_bits<M>(key[i], g.n);
+        const uint32_t counted = g.score_mode == 0 ? bits : 0xFFu;
+        if (mk) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if ((counted >> j) & 1u) acc += fixed_point_score(key[i][j], e_max);
+        }
         uint32_t word = bits << (8 * (lane & 3));
         word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
         word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
         if ((lane & 3) == 0 && in_kp) nm_bits[row * g.wpr + (k0 >> 5)] = word;
     }
-    if (in_kp && acc) atomicAdd(&s_score[(int)(k0 / g.bk) - first_blk], acc);
+    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
+    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
+    if ((lane & 3) == 0 && in_kp && acc) atomicAdd(&s_score[(int)(k0 / g.bk) - first_blk], acc);
     __syncthreads();
     if (threadIdx.x < kM1ChunkK / 32 + 2) {
         const int jb = first_blk + threadIdx.x;
@@ -140,8 +209,9 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
     }
 }
 
-// One CTA per row tile: rank the block scores, emit the kept columns in ascending order and
-// clear the mask words of pruned blocks.
+// K-M2.  grid = (row tiles, block_rows / 32).  Every CTA ranks its row tile's block scores (cheap)
+// and clears the mask words of pruned blocks in its own 32 rows; the CTA with blockIdx.y == 0 also
+// emits the kept columns in ascending order.
 __global__ void __launch_bounds__(256)
 block_select_kernel(Geometry g, const unsigned long long *__restrict__ score,
                     int32_t *__restrict__ blk_col, uint32_t *__restrict__ nm_bits) {
@@ -164,33 +234,33 @@ block_select_kernel(Geometry g, const unsigned long long *__restrict__ score,
         kept[j] = rank < g.kkeep;
     }
     __syncthreads();
-    // ascending compaction: block-wide exclusive scan over chunks of blockDim.x flags
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int j0 = 0; j0 < g.nblk; j0 += blockDim.x) {
-        const int j = j0 + threadIdx.x;
-        const int f = (j < g.nblk) ? kept[j] : 0;
-        const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, f);
-        const int before = __popc(ballot & ((1u << lane) - 1u));
-        if (lane == 0) s_warp_tot[warp] = __popc(ballot);
-        __syncthreads();
-        int warp_off = 0, tot = 0;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
-            if (w < warp) warp_off += s_warp_tot[w];
-            tot += s_warp_tot[w];
+    if (blockIdx.y == 0) {
+        // ascending compaction: block-wide exclusive scan over chunks of blockDim.x flags
+        for (int j0 = 0; j0 < g.nblk; j0 += blockDim.x) {
+            const int j = j0 + threadIdx.x;
+            const int f = (j < g.nblk) ? kept[j] : 0;
+            const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, f);
+            const int before = __popc(ballot & ((1u << lane) - 1u));
+            if (lane == 0) s_warp_tot[warp] = __popc(ballot);
+            __syncthreads();
+            int warp_off = 0, tot = 0;
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+                if (w < warp) warp_off += s_warp_tot[w];
+                tot += s_warp_tot[w];
+            }
+            if (f) blk_col[(int64_t)rt * g.kkeep + s_base + warp_off + before] = j;
+            __syncthreads();
+            if (threadIdx.x == 0) s_base += tot;
+            __syncthreads();
         }
-        if (f) blk_col[(int64_t)rt * g.kkeep + s_base + warp_off + before] = j;
-        __syncthreads();
-        if (threadIdx.x == 0) s_base += tot;
-        __syncthreads();
     }
-    // final mask = group bits AND block kept
+    // final mask = group bits AND block kept: one warp per row, lanes stride over the row's words
     const int wpb = g.bk / 32;
-    const int64_t items = (int64_t)g.nblk * g.bm * wpb;
-    for (int64_t i = threadIdx.x; i < items; i += blockDim.x) {
-        const int w = (int)(i % wpb);
-        const int r = (int)((i / wpb) % g.bm);
-        const int jb = (int)(i / ((int64_t)wpb * g.bm));
-        if (!kept[jb]) nm_bits[((int64_t)rt * g.bm + r) * g.wpr + jb * wpb + w] = 0u;
+    for (int r = warp; r < 32; r += 8) {
+        uint32_t *row_words = nm_bits + ((int64_t)rt * g.bm + blockIdx.y * 32 + r) * g.wpr;
+        for (int wc = lane; wc < g.wpr; wc += 32)
+            if (!kept[wc / wpb]) row_words[wc] = 0u;
     }
 }
 
@@ -211,19 +281,19 @@ cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, i
     if (e != cudaSuccess) return e;
     const bool vec_ok = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_s) & 15u) == 0);
 
-    const int64_t items = (int64_t)g.rows * ((g.k + 7) / 8);
-    int grid0 = (int)((items + 255) / 256 < 148 * 8 ? (items + 255) / 256 : 148 * 8);
+    const int64_t items = (int64_t)g.rows * ((g.k + 1023) / 1024);     // one warp per item
+    int grid0 = (int)((items + 7) / 8 < 148 * 8 ? (items + 7) / 8 : 148 * 8);
     if (grid0 < 1) grid0 = 1;
     max_key_kernel<<<grid0, 256, 0, st>>>(d_s, ld, g.rows, g.k, vec_ok, max_key);
 
-    dim3 grid1((unsigned)((g.kp() + kM1ChunkK - 1) / kM1ChunkK), (unsigned)g.nrt);
+    dim3 grid1((unsigned)(g.mp() / kM1Rows), (unsigned)((g.kp() + kM1ChunkK - 1) / kM1ChunkK));
     if (g.m == 4)
         group_select_kernel<4><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
     else
         group_select_kernel<8><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
 
     const size_t smem = (size_t)g.nblk * (sizeof(unsigned long long) + sizeof(int));
-    block_select_kernel<<<g.nrt, 256, smem, st>>>(g, score, d_blk_col, d_nm_bits);
+    block_select_kernel<<<dim3((unsigned)g.nrt, (unsigned)(g.bm / 32)), 256, smem, st>>>(g, score, d_blk_col, d_nm_bits);
     return cudaGetLastError();
 }
 

@@ -40,6 +40,8 @@ struct TcParams {
     int nst, wcap, bk, n_col_tiles, num_tiles, rows;
     int64_t ncols;
     uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
+    int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
+    int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -81,6 +83,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile(
@@ -168,7 +175,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // between 8-row K groups and box_bytes between 64-column groups.
 template <int NT, bool kSparse, int kAccStages, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
-spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, TcParams p) {
+spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
+               const __grid_constant__ CUtensorMap map_a, TcParams p) {
     constexpr int kTileN = NT * kBoxN;
     constexpr int kMetaCols = kSparse ? 8 : 0;                       // two 4-column metadata buffers
     constexpr int kTmemCols = (kAccStages * kTileN + kMetaCols) <= 256 ? 256 : 512;
@@ -218,12 +226,23 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) break;
                     const uint32_t dst = ring + s * p.stage_bytes;
                     mbar_expect_tx(bar_full + 8 * s, tx_bytes);
-                    bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, bar_full + 8 * s);
+                    // untiled bulk copies are served one at a time (~0.3 us each, whatever their size);
+                    // tiled loads pipeline, so the weight tile is fetched as a box of 256-byte rows
+                    if (p.a_map)
+                        tma_load_2d(dst, &map_a, 0, (int)((((int64_t)st * p.wcap + e) * p.entry_bytes) >> 8), bar_full + 8 * s);
+                    else
+                        bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, bar_full + 8 * s);
                     const int krow = cols[e] * p.bk;
+                    if (p.x_map_3d) {
+                        // each copy instruction costs the issuing thread far more than its share of the
+                        // transfer, so the NT boxes of X come in with a single 3-D load
+                        tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, bar_full + 8 * s);
+                    } else {
 #pragma unroll
-                    for (int b = 0; b < NT; ++b)
-                        tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow,
-                                    bar_full + 8 * s);
+                        for (int b = 0; b < NT; ++b)
+                            tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow,
+                                        bar_full + 8 * s);
+                    }
                     if (++s == p.num_stages) { s = 0; ph ^= 1u; }
                 }
             }
@@ -360,111 +379,159 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 // --------------------------------------------------------------------- execution image kernels
 
 // Union walk of the r = 128 / bm row tiles that share one CTA tile: ascending block columns.
-__global__ void build_walk_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int wcap,
-                                  int32_t *__restrict__ walk_col, int32_t *__restrict__ walk_len) {
-    const int st = blockIdx.x * blockDim.x + threadIdx.x;
-    const int nst = (g.nrt + r - 1) / r;
-    if (st >= nst) return;
-    int pos[4] = {0, 0, 0, 0};
-    int len = 0;
-    for (;;) {
-        int best = 0x7FFFFFFF;
-        for (int i = 0; i < r; ++i) {
-            const int rt = st * r + i;
-            if (rt < g.nrt && pos[i] < g.kkeep) best = min(best, blk_col[(int64_t)rt * g.kkeep + pos[i]]);
-        }
-        if (best == 0x7FFFFFFF) break;
-        for (int i = 0; i < r; ++i) {
-            const int rt = st * r + i;
-            if (rt < g.nrt && pos[i] < g.kkeep && blk_col[(int64_t)rt * g.kkeep + pos[i]] == best) ++pos[i];
-        }
-        walk_col[(int64_t)st * wcap + len++] = best;
+// One CTA per CTA tile: mark the kept columns in a shared bitmap, then compact it.
+__global__ void __launch_bounds__(128)
+build_walk_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int wcap,
+                  int32_t *__restrict__ walk_col, int32_t *__restrict__ walk_len) {
+    __shared__ uint32_t s_bits[128];                 // nblk <= 4096
+    __shared__ int s_prefix[129];
+    const int st = blockIdx.x;
+    const int words = (g.nblk + 31) / 32;
+    for (int i = threadIdx.x; i < words; i += blockDim.x) s_bits[i] = 0u;
+    __syncthreads();
+    const int first_rt = st * r;
+    const int n_rt = min(r, g.nrt - first_rt);
+    for (int i = threadIdx.x; i < n_rt * g.kkeep; i += blockDim.x) {
+        const int jb = blk_col[(int64_t)first_rt * g.kkeep + i];
+        atomicOr(&s_bits[jb >> 5], 1u << (jb & 31));
     }
-    walk_len[st] = len;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int i = 0; i < words; ++i) { s_prefix[i] = run; run += __popc(s_bits[i]); }
+        s_prefix[words] = run;
+        walk_len[st] = run;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < words; i += blockDim.x) {
+        uint32_t b = s_bits[i];
+        int o = s_prefix[i];
+        while (b) {
+            const int t = __ffs(b) - 1;
+            b &= b - 1;
+            walk_col[(int64_t)st * wcap + o++] = i * 32 + t;
+        }
+    }
 }
 
-// One CTA per kept block: scatter its values into the (pre-zeroed) tile of its walk entry.
+// One CTA per walk entry: assemble the entry's weight tile (and 2:4 metadata) in shared memory from
+// the canonical values and offsets of the row tiles that keep this block column, zeros for row tiles
+// that do not, then write it out with coalesced 16-byte stores.
 // Dense image: element (row, k) of the tile at [k/8][row][k%8].
-// Sparse image: per 4-group two slots (ascending position, zero-padded), slot pair p = k/4 stored at
-// compressed column 2p + slot, same [c/8][row][c%8] layout; metadata word j = k/32 of row L' holds
-// 16 bits for row (16*(row/16) + row%8) and 16 bits for that row + 8, where
-// L' = row%8 + 8*((k/16)%2) + 16*(row/16); nibble g%4... of a 4-group = idx0 | idx1 << 2.
+// Sparse image: per aligned 4-group two slots (ascending position, zero-padded); slot pair of group
+// q stored at compressed columns 2q, 2q+1 in the same [c/8][row][c%8] layout.  Metadata (2048 bytes):
+// 16-byte row L = row%8 + 8*((k/16)%2) + 16*(row/16), 32-bit word k/32, nibble of the 4-group at bit
+// (k%16) + 16*((row/8)%2), value idx0 | idx1 << 2.
 template <bool kSparse>
 __global__ void __launch_bounds__(256)
 build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16_t *__restrict__ vals,
                    const uint32_t *__restrict__ idx, int r, int wcap, const int32_t *__restrict__ walk_col,
                    const int32_t *__restrict__ walk_len, uint32_t a_bytes, uint32_t entry_bytes,
                    uint8_t *__restrict__ image) {
-    const int blk = blockIdx.x;
-    const int rt = blk / g.kkeep;
-    const int jb = blk_col[blk];
-    const int st = rt / r;
-    __shared__ int s_entry;
-    if (threadIdx.x == 0) {
-        int lo = 0, hi = walk_len[st] - 1, found = 0;
-        const int32_t *wc = walk_col + (int64_t)st * wcap;
-        while (lo <= hi) {
-            const int mid = (lo + hi) >> 1;
-            if (wc[mid] == jb) { found = mid; break; }
-            if (wc[mid] < jb) lo = mid + 1; else hi = mid - 1;
+    extern __shared__ uint4 s_tile4[];
+    uint8_t *tile = reinterpret_cast<uint8_t *>(s_tile4);
+    __shared__ int s_blk[4];
+    const int st = blockIdx.x / wcap, e = blockIdx.x - st * wcap;
+    if (e >= walk_len[st]) return;
+    const int jb = walk_col[(int64_t)st * wcap + e];
+    for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) s_tile4[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x < r) {
+        // does row tile st*r + threadIdx.x keep block column jb, and in which slot?
+        const int rt = st * r + threadIdx.x;
+        int found = -1;
+        if (rt < g.nrt) {
+            const int32_t *bc = blk_col + (int64_t)rt * g.kkeep;
+            int lo = 0, hi = g.kkeep - 1;
+            while (lo <= hi) {
+                const int mid = (lo + hi) >> 1;
+                const int v = bc[mid];
+                if (v == jb) { found = rt * g.kkeep + mid; break; }
+                if (v < jb) lo = mid + 1; else hi = mid - 1;
+            }
         }
-        s_entry = found;
+        s_blk[threadIdx.x] = found;
     }
     __syncthreads();
-    uint8_t *tile = image + ((int64_t)st * wcap + s_entry) * entry_bytes;
-    const int row0 = (rt % r) * g.bm;
     const int groups = g.groups();
-    const int64_t vpb = g.vals_per_block();
-    const uint16_t *vb = vals + (int64_t)blk * vpb;
-    const uint32_t *ib = idx + (int64_t)blk * (vpb * g.idx_bits / 32);
+    const int vpb = (int)g.vals_per_block();
+    const int idx_words = vpb * g.idx_bits / 32;
     const uint32_t field = (1u << g.idx_bits) - 1u;
-    if constexpr (!kSparse) {
-        for (int o = threadIdx.x; o < (int)vpb; o += blockDim.x) {
-            const int item = o / g.n;
-            const int lr = item / groups, gi = item - lr * groups;
-            const int bit = o * g.idx_bits;
-            uint32_t t = ib[bit >> 5] >> (bit & 31);
-            if ((bit & 31) + g.idx_bits > 32) t |= ib[(bit >> 5) + 1] << (32 - (bit & 31));
-            t &= field;
-            const int k = gi * g.m + (int)t, row = row0 + lr;
-            *reinterpret_cast<uint16_t *>(tile + (k >> 3) * 2048 + row * 16 + (k & 7) * 2) = vb[o];
+    // canonical values and offsets of one kept block, staged with coalesced 16-byte loads
+    uint16_t *vb = reinterpret_cast<uint16_t *>(tile + entry_bytes);
+    uint32_t *ib = reinterpret_cast<uint32_t *>(tile + entry_bytes + (size_t)vpb * 2);
+    for (int sub = 0; sub < r; ++sub) {
+        const int blk = s_blk[sub];
+        if (blk < 0) continue;
+        const int row0 = sub * g.bm;
+        __syncthreads();
+        {
+            const uint4 *vsrc = reinterpret_cast<const uint4 *>(vals + (int64_t)blk * vpb);      // vpb*2 is a multiple of 64
+            for (int i = threadIdx.x; i < vpb / 8; i += blockDim.x) reinterpret_cast<uint4 *>(vb)[i] = __ldg(vsrc + i);
+            const uint32_t *isrc = idx + (int64_t)blk * idx_words;
+            for (int i = threadIdx.x; i < idx_words; i += blockDim.x) ib[i] = __ldg(isrc + i);
         }
-    } else {
-        // one thread per (local row, 4-group): at most two kept values by construction
-        const int quads = g.bk / 4;
-        uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
-        for (int item = threadIdx.x; item < g.bm * quads; item += blockDim.x) {
-            const int lr = item / quads, qd = item - lr * quads;
-            const int row = row0 + lr;
-            // kept values of this row whose position falls into [4*qd, 4*qd+4)
-            const int gi = (qd * 4) / g.m;
-            uint16_t v[2] = {0, 0};
-            int pos[2] = {0, 0}, cnt = 0;
-            for (int vv = 0; vv < g.n; ++vv) {
-                const int o = (lr * groups + gi) * g.n + vv;
+        __syncthreads();
+        if constexpr (!kSparse) {
+            for (int o = threadIdx.x; o < vpb; o += blockDim.x) {
+                const int item = o / g.n;
+                const int lr = item / groups, gi = item - lr * groups;
                 const int bit = o * g.idx_bits;
                 uint32_t t = ib[bit >> 5] >> (bit & 31);
                 if ((bit & 31) + g.idx_bits > 32) t |= ib[(bit >> 5) + 1] << (32 - (bit & 31));
                 t &= field;
-                const int k = gi * g.m + (int)t;
-                if ((k >> 2) == qd && cnt < 2) { v[cnt] = vb[o]; pos[cnt] = k & 3; ++cnt; }
+                const int k = gi * g.m + (int)t, row = row0 + lr;
+                *reinterpret_cast<uint16_t *>(tile + (k >> 3) * 2048 + row * 16 + (k & 7) * 2) = vb[o];
             }
-            if (cnt == 0) { pos[0] = 0; pos[1] = 1; }
-            else if (cnt == 1) {
-                if (pos[0] == 3) { v[1] = v[0]; v[0] = 0; pos[1] = 3; pos[0] = 0; }
-                else pos[1] = 3;
+        } else {
+            // one thread per (local row, 4-group): at most two kept values by construction
+            const int quads = g.bk / 4;
+            uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
+            for (int item = threadIdx.x; item < g.bm * quads; item += blockDim.x) {
+                const int lr = item / quads, qd = item - lr * quads;
+                const int row = row0 + lr;
+                const int gi = (qd * 4) / g.m;
+                uint16_t v[2] = {0, 0};
+                int pos[2] = {0, 0}, cnt = 0;
+                for (int vv = 0; vv < g.n; ++vv) {
+                    const int o = (lr * groups + gi) * g.n + vv;
+                    const int bit = o * g.idx_bits;
+                    uint32_t t = ib[bit >> 5] >> (bit & 31);
+                    if ((bit & 31) + g.idx_bits > 32) t |= ib[(bit >> 5) + 1] << (32 - (bit & 31));
+                    t &= field;
+                    const int k = gi * g.m + (int)t;
+                    if ((k >> 2) == qd && cnt < 2) { v[cnt] = vb[o]; pos[cnt] = k & 3; ++cnt; }
+                }
+                if (cnt == 0) { pos[0] = 0; pos[1] = 1; }
+                else if (cnt == 1) {
+                    if (pos[0] == 3) { v[1] = v[0]; v[0] = 0; pos[1] = 3; pos[0] = 0; }
+                    else pos[1] = 3;
+                }
+                const int c0 = 2 * qd;                       // even: both slots share one 16-byte chunk
+                *reinterpret_cast<uint32_t *>(tile + (c0 >> 3) * 2048 + row * 16 + (c0 & 7) * 2) =
+                    (uint32_t)v[0] | ((uint32_t)v[1] << 16);
+                const uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
+                const int k0 = qd * 4;
+                const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
+                atomicOr(&meta[lrow * 4 + (k0 >> 5)], nib << ((k0 & 15) + 16 * ((row >> 3) & 1)));
             }
-            const int c0 = 2 * qd;
-            *reinterpret_cast<uint16_t *>(tile + (c0 >> 3) * 2048 + row * 16 + (c0 & 7) * 2) = v[0];
-            *reinterpret_cast<uint16_t *>(tile + ((c0 + 1) >> 3) * 2048 + row * 16 + ((c0 + 1) & 7) * 2) = v[1];
-            const uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
-            const int k0 = qd * 4;
-            const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
-            const int word = k0 >> 5;
-            const int shift = (k0 & 15) + 16 * ((row >> 3) & 1);
-            atomicOr(&meta[lrow * 4 + word], nib << shift);
         }
     }
+    if constexpr (kSparse) {
+        // row tiles that do not keep this block still need valid (distinct, ascending) index pairs
+        uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
+        for (int sub = 0; sub < r; ++sub) {
+            if (s_blk[sub] >= 0) continue;
+            for (int item = threadIdx.x; item < g.bm * (g.bk / 4); item += blockDim.x) {
+                const int lr = item / (g.bk / 4), qd = item - lr * (g.bk / 4);
+                const int row = sub * g.bm + lr, k0 = qd * 4;
+                const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
+                atomicOr(&meta[lrow * 4 + (k0 >> 5)], 0x4u << ((k0 & 15) + 16 * ((row >> 3) & 1)));
+            }
+        }
+    }
+    __syncthreads();
+    uint4 *out = reinterpret_cast<uint4 *>(image + ((int64_t)st * wcap + e) * entry_bytes);
+    for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = s_tile4[i];
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -498,9 +565,36 @@ bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// X viewed as [ncols/64][k][64] (needs ncols % 64 == 0): box = 64 columns x bk rows x nt column groups,
+// which lands in shared memory exactly like nt consecutive 2-D boxes.
+bool make_map_x3d(CUtensorMap *map, const void *base, uint64_t ncols, uint64_t k, uint64_t ldx, uint32_t bk, uint32_t nt) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kBoxN, k, ncols / kBoxN};
+    cuuint64_t strides[2] = {ldx * 2ull, (cuuint64_t)kBoxN * 2ull};
+    cuuint32_t box[3] = {(cuuint32_t)kBoxN, bk, nt};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The execution image as a matrix of 256-byte rows; one box = one walk entry (weight tile + metadata).
+bool make_map_image(CUtensorMap *map, const void *image, uint64_t total_bytes, uint32_t entry_bytes) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || entry_bytes % 256 != 0 || entry_bytes / 256 > 256 || total_bytes / 256 >= (1ull << 31)) return false;
+    cuuint64_t dims[2] = {256, total_bytes / 256};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {256, entry_bytes / 256};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(image), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int NT, bool kSparse, int kAccStages, typename OutT>
-cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const TcParams &p, int grid, size_t smem,
-                           cudaStream_t st) {
+cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const CUtensorMap &ma, const TcParams &p,
+                           int grid, size_t smem, cudaStream_t st) {
     auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT>;
     static size_t configured = 0;                       // largest dynamic shared memory opted into so far
     if (smem > configured) {
@@ -508,7 +602,7 @@ cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const T
         if (e != cudaSuccess) return e;
         configured = smem;
     }
-    kern<<<grid, kThreads, smem, st>>>(mx, my, p);
+    kern<<<grid, kThreads, smem, st>>>(mx, my, ma, p);
     return cudaGetLastError();
 }
 
@@ -540,15 +634,20 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
     int32_t *walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
     int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
     uint8_t *image = d_exec + L.image_off;
-    cudaError_t e = cudaMemsetAsync(image, 0, (size_t)L.nst * L.wcap * L.entry_bytes, st);
-    if (e != cudaSuccess) return e;
-    build_walk_kernel<<<(L.nst + 127) / 128, 128, 0, st>>>(g, d_blk_col, L.r, L.wcap, walk_col, walk_len);
+    build_walk_kernel<<<L.nst, 128, 0, st>>>(g, d_blk_col, L.r, L.wcap, walk_col, walk_len);
+    const int grid = L.nst * L.wcap;
+    const size_t smem_img = (size_t)L.entry_bytes + (size_t)g.vals_per_block() * 2 + (size_t)(g.vals_per_block() * g.idx_bits / 32) * 4 + 16;
+    if (smem_img > 48 * 1024) {      // large blocks with many kept values need the opt-in shared memory size
+        cudaError_t e = sparse ? cudaFuncSetAttribute(build_image_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_img)
+                               : cudaFuncSetAttribute(build_image_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_img);
+        if (e != cudaSuccess) return e;
+    }
     if (sparse)
-        build_image_kernel<true><<<g.nrt * g.kkeep, 256, 0, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
-                                                                   walk_len, L.a_bytes, L.entry_bytes, image);
-    else
-        build_image_kernel<false><<<g.nrt * g.kkeep, 256, 0, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
+        build_image_kernel<true><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
                                                                     walk_len, L.a_bytes, L.entry_bytes, image);
+    else
+        build_image_kernel<false><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
+                                                                     walk_len, L.a_bytes, L.entry_bytes, image);
     return cudaGetLastError();
 }
 
@@ -570,8 +669,10 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (sm_count <= 0) sm_count = 148;
     }
-    // column tile: 4 boxes (256 columns) when two accumulators fit beside the metadata, else 3
-    int nt = (nt_override >= 1 && nt_override <= 4) ? nt_override : (sparse ? 3 : 4);
+    // column tile: 4 boxes (256 columns).  For the sparse image that leaves room for one accumulator
+    // only (256 + 8 metadata columns), which still beats 3 boxes with two accumulators: the kernel is
+    // bound by bytes into shared memory, and wider tiles amortise the weight tile over more columns.
+    int nt = (nt_override >= 1 && nt_override <= 4) ? nt_override : 4;
     const int64_t boxes = (ncols + kBoxN - 1) / kBoxN;
     if (boxes < nt) nt = (int)boxes;
     TcParams p;
@@ -594,9 +695,13 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.num_stages = stages;
     const size_t smem = (size_t)stages * p.stage_bytes + fixed + 1024;
 
-    CUtensorMap mx, my;
-    if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, (uint64_t)ncols, (uint64_t)g.k, (uint64_t)ldx,
-                     kBoxN, (uint32_t)g.bk))
+    CUtensorMap mx, my, ma;
+    p.a_map = make_map_image(&ma, p.image, (uint64_t)L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
+    if (!p.a_map) ma = CUtensorMap{};
+    p.x_map_3d = (ncols % kBoxN == 0) &&
+                 make_map_x3d(&mx, d_x, (uint64_t)ncols, (uint64_t)g.k, (uint64_t)ldx, (uint32_t)g.bk, (uint32_t)nt);
+    if (!p.x_map_3d && !make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, (uint64_t)ncols, (uint64_t)g.k,
+                                    (uint64_t)ldx, kBoxN, (uint32_t)g.bk))
         return cudaErrorInvalidValue;
     const bool f32 = y_dtype != 0;
     if (!make_map_2d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, f32 ? 4 : 2, d_y,
@@ -605,8 +710,8 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
 
 #define CRISP_TC_LAUNCH(NTV, SP, ACC)                                                                     \
-    (f32 ? launch_variant<NTV, SP, ACC, float>(mx, my, p, grid, smem, st)                                 \
-         : launch_variant<NTV, SP, ACC, uint16_t>(mx, my, p, grid, smem, st))
+    (f32 ? launch_variant<NTV, SP, ACC, float>(mx, my, ma, p, grid, smem, st)                                 \
+         : launch_variant<NTV, SP, ACC, uint16_t>(mx, my, ma, p, grid, smem, st))
     if (sparse) {
         switch (nt) {
             case 1: return CRISP_TC_LAUNCH(1, true, 2);
