@@ -134,7 +134,7 @@ def oracle_sample_cols(layer, w, s, x, target_s=12.0):
     t0 = time.perf_counter()
     oracle.spmm_fp64(wd, probe)
     per_col = (time.perf_counter() - t0) / pc
-    return int(max(4, min(x.shape[1], target_s / max(per_col, 1e-9))))
+    return int(max(4, min(x.shape[1], 1024, target_s / max(per_col, 1e-9))))
 
 
 def run_reference(args, layer, rank):
@@ -166,6 +166,85 @@ def run_reference(args, layer, rank):
 
 
 # ---------------------------------------------------------------------------- GPU arm
+
+def roofline_terms(model, peaks, spmm_ms, ncols):
+    """Slot-aware tensor time and algorithmic-byte HBM time of one crisp_spmm call."""
+    useful = 2.0 * model["nnz"] * ncols
+    slot_flops = 2.0 * model["slot_macs"]
+    hbm_bytes = model["vals_bytes"] + model["idx_bytes"] + model["blk_col_bytes"] + model["x_bytes"] + model["y_bytes"]
+    t_tensor = slot_flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = hbm_bytes / (peaks["hbm_gbs"] * 1e9)
+    return {"useful_flops": useful, "slot_flops": slot_flops, "hbm_bytes": hbm_bytes, "t_tensor": t_tensor,
+            "t_hbm": t_hbm, "frac": max(t_tensor, t_hbm) / (spmm_ms * 1e-3),
+            "frac_literal": max(useful / (peaks["bf16_tflops"] * 1e12), t_hbm) / (spmm_ms * 1e-3)}
+
+
+CELL_WORKLOADS = ["sweep_2:4_keep1.0", "sweep_2:4_keep0.25", "sweep_2:4_keep0.1", "sweep_1:4_keep0.5",
+                  "sweep_2:8_keep0.5", "sweep_4:8_keep0.5", "config2"]
+
+
+def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=12):
+    """SpMM-only timings of further cells of the metric (same protocol: events, L2 flushed between
+    iterations), each beside a dense bf16 cuBLAS GEMM of the same shape."""
+    out = []
+    stream = torch.cuda.current_stream()
+    for name in CELL_WORKLOADS:
+        layer = pick_layer(name)
+        if name.startswith("sweep_"):
+            d_s, d_w, d_x = shared                      # every sweep cell prunes the same W / S / X
+        else:
+            w, s, x = wl.make_layer_inputs(layer)
+            d_s = torch.from_numpy(s).to(dev)
+            d_w = torch.from_numpy(w.view(np.int16)).to(dev).view(torch.bfloat16)
+            d_x = torch.from_numpy(x.view(np.int16)).to(dev).view(torch.bfloat16)
+        d_y = torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16, device=dev)
+        L = B.HybridLayer(layer.rows, layer.k, layer.n, layer.m, layer.block_rows, layer.block_k,
+                          layer.keep_ratio, device=dev)
+        L.build_mask(d_s).encode(d_w)
+        ts, td = [], []
+        for i in range(3 + iters):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            L.spmm(d_x, y=d_y)
+            b.record(stream)
+            flush_l2()
+            c, d = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c.record(stream)
+            torch.matmul(d_w, d_x, out=d_y)
+            d.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b)); td.append(c.elapsed_time(d))
+        model = L.bytes_model(layer.ncols)
+        ms = float(np.mean(ts))
+        r = roofline_terms(model, peaks, ms, layer.ncols)
+        out.append({"workload": name, "kernel": B.PATH_NAMES[model["path"]], "kkeep": L.kkeep,
+                    "spmm_us": ms * 1e3, "dense_cublas_us": float(np.mean(td)) * 1e3,
+                    "speedup_vs_dense_cublas": float(np.mean(td)) / ms,
+                    "useful_tflops": r["useful_flops"] / (ms * 1e-3) / 1e12,
+                    "t_tensor_us": r["t_tensor"] * 1e6, "t_hbm_us": r["t_hbm"] * 1e6,
+                    "roofline_frac": r["frac"], "roofline_frac_literal": r["frac_literal"],
+                    "device_status": L.device_status()})
+        L.close()
+    return out
+
+
+def recorded_traffic(workload, kernel):
+    """DRAM bytes per launch from the committed ncu capture, or None when the kernel source has
+    changed since the counters were taken."""
+    import hashlib
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return None
+    rec = json.load(open(p))
+    src = os.path.join(ROOT, "paper_2311_14272_b200", "csrc", "spmm_tc.cu")
+    sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    for r in rec.get("captures", []):
+        if r["workload"] == workload and r["kernel"] == kernel and r["source_sha256"] == sha:
+            return r["dram_bytes_per_launch"]
+    return None
+
 
 def run_ours(args, layer, rank, world):
     import torch
@@ -302,7 +381,7 @@ def run_ours(args, layer, rank, world):
     else:
         roof = {"bound": "hbm", "achieved": hbm_bytes / (spmm_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update({"traffic": None, "peak_kind": f"of {peak_kind} (burst)", "kernel": B.PATH_NAMES[model["path"]],
+    roof.update({"traffic": recorded_traffic(args.workload, B.PATH_NAMES[model["path"]]), "peak_kind": f"of {peak_kind} (burst)", "kernel": B.PATH_NAMES[model["path"]],
                  "t_tensor_us": t_tensor * 1e6, "t_hbm_us": t_hbm * 1e6, "t_kernel_us": spmm_ms * 1e3,
                  "frac_of_max_roof": max(t_tensor, t_hbm) / (spmm_ms * 1e-3),
                  "frac_literal_useful_flops": useful_flops / (spmm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
@@ -329,9 +408,11 @@ def run_ours(args, layer, rank, world):
            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
                    "h2d_bytes_per_step": int(h_s.numel() * 4 + h_w.numel() * 2 + h_x.numel() * 2),
                    "d2h_bytes_per_step": int(h_y.numel() * 2)},
-           "gpu_launches": 5 * args.steps, "kernels_per_step": {"mask": 3, "encode": 1, "spmm": 1},
+           "gpu_launches": 7 * args.steps, "kernels_per_step": {"mask": 3, "encode": 3, "spmm": 1},
            "clocks": clocks, "roofline": roof, "phases": phases, "device_status": status}
 
+    if rank == 0 and world == 1 and not args.no_cells and args.workload.startswith("sweep_"):
+        out["cells"] = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)
@@ -355,6 +436,7 @@ def main():
     ap.add_argument("--workload", default="sweep_2:4_keep0.5",
                     help="sweep_<n>:<m>_keep<r> (4096x4096x8192, block 128x64), config1 or config2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cells", action="store_true", help="skip the extra SpMM-only cells")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
