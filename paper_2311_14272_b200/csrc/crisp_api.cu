@@ -240,7 +240,13 @@ crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ld
         e = crisp::launch_spmm_direct(h->g, h->d_blk_col, h->d_vals, h->d_idx, d_x_bf16, ldx, ncols,
                                       d_y, ldy, y_dtype, (cudaStream_t)stream);
     } else {
+        const char *pair = std::getenv("CRISP_TC_PAIR");   // 1: CTA-pair kernel, 0: single-CTA kernel
+        const bool use_pair = pair && std::atoi(pair) == 1 && crisp::tc_pair_supported(h->g, ncols);
         const char *nt = std::getenv("CRISP_TC_NT");     // column boxes per CTA tile, tuning only
+        if (use_pair)
+            e = crisp::launch_spmm_tc_pair(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx,
+                                           ncols, d_y, ldy, y_dtype, (cudaStream_t)stream);
+        else
         e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx, ncols,
                                   d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, (cudaStream_t)stream);
     }

@@ -74,6 +74,9 @@ struct TcImageLayout {
     uint32_t a_bytes;       // weight tile bytes per walk entry
     uint32_t entry_bytes;   // weight tile + metadata
     size_t walk_col_off, walk_len_off, image_off, total_bytes;   // offsets inside the exec payload
+    int npairs;             // pairs of adjacent CTA tiles (CTA-pair kernel)
+    int pwcap;              // capacity of one pair's union walk list
+    size_t pair_col_off, pair_len_off, pair_src_off;
 };
 bool tc_pattern_is_sparse(const Geometry &g);
 TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
@@ -83,6 +86,11 @@ bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int 
 cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
                            const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
                            int nt_override, cudaStream_t st);
+// spmm_tc_pair.cu: two CTAs (cta_group::2) share the X tile of the union of two adjacent CTA tiles' lists
+bool tc_pair_supported(const Geometry &g, int64_t ncols);
+cudaError_t launch_spmm_tc_pair(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
+                                const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy,
+                                int y_dtype, cudaStream_t st);
 
 // spmm_direct.cu
 cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
