@@ -45,27 +45,33 @@ CASES = [
     (64, 96, 50, 8, 8, 32, 32, 0.67),
     (130, 384, 96, 2, 4, 128, 128, 0.34),
     (64, 288, 40, 3, 8, 64, 96, 0.67),
+    (384, 768, 576, 2, 4, 128, 64, 0.5),     # 3 CTA tiles (odd: one pair has a ghost side), 2.25 column tiles
+    (512, 512, 320, 1, 4, 64, 64, 0.25),
+    (256, 256, 128, 2, 8, 32, 32, 0.5),
 ]
 
 
 # which execution image crisp_encode lays out: the default choice (2:4 sparse MMA when n <= 2, dense
 # tiles otherwise), dense tiles forced, or none (CUDA-core kernel on the canonical format)
-IMAGES = ["auto", "dense", "none"]
+# "pair" / "dense-pair": same images, run by the CTA-pair kernel where the shape allows it
+IMAGES = ["auto", "dense", "none", "pair", "dense-pair"]
 
 
 @pytest.fixture(params=IMAGES)
 def image(request, monkeypatch):
-    if request.param == "auto":
+    kind = request.param
+    monkeypatch.setenv("CRISP_TC_PAIR", "1" if kind.endswith("pair") else "0")
+    if kind in ("auto", "pair"):
         monkeypatch.delenv("CRISP_EXEC_IMAGE", raising=False)
     else:
-        monkeypatch.setenv("CRISP_EXEC_IMAGE", request.param)
-    return request.param
+        monkeypatch.setenv("CRISP_EXEC_IMAGE", "dense" if kind.startswith("dense") else kind)
+    return kind
 
 
 def expected_path(B, image, n, kkeep=1):
     if image == "none":
         return B.PATH_DIRECT
-    if image == "dense":
+    if image.startswith("dense"):
         return B.PATH_DENSE
     return B.PATH_SPARSE if n <= 2 else B.PATH_DENSE
 
