@@ -95,29 +95,42 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int len = p.walk_len[st];
                 const int32_t *cols = p.walk_col + (int64_t)st * p.wcap;
                 const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
-                for (int e = 0; e < len; ++e) {
-                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) break;
-                    const uint32_t dst = ring + s * p.stage_bytes;
-                    mbar_expect_tx(bar_full + 8 * s, tx_bytes);
-                    // untiled bulk copies are served one at a time (~0.3 us each, whatever their size);
-                    // tiled loads pipeline, so the weight tile is fetched as a box of 256-byte rows
-                    if (p.a_map)
-                        tma_load_2d(dst, &map_a, 0, (int)((((int64_t)st * p.wcap + e) * p.entry_bytes) >> 8), bar_full + 8 * s);
-                    else
-                        bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, bar_full + 8 * s);
-                    const int krow = cols[e] * p.bk;
-                    if (p.x_map_3d) {
-                        // each copy instruction costs the issuing thread far more than its share of the
-                        // transfer, so the NT boxes of X come in with a single 3-D load
-                        tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, bar_full + 8 * s);
-                    } else {
+                // The block column of entry e is a global load in this thread's serial loop; left where it
+                // is used it costs one L2 round trip (~0.4 us) per stage.  Keep the next four in registers.
+                int col_q[4];
 #pragma unroll
-                        for (int b = 0; b < NT; ++b)
-                            tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow,
+                for (int u = 0; u < 4; ++u) col_q[u] = u < len ? __ldg(cols + u) : 0;
+                bool ok = true;
+                for (int e0 = 0; e0 < len && ok; e0 += 4) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int e = e0 + u;
+                        if (e >= len) break;
+                        const int krow = col_q[u] * p.bk;
+                        if (e + 4 < len) col_q[u] = __ldg(cols + e + 4);
+                        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t dst = ring + s * p.stage_bytes;
+                        mbar_expect_tx(bar_full + 8 * s, tx_bytes);
+                        // untiled bulk copies are served one at a time; tiled loads pipeline, so the weight
+                        // tile is fetched as a box of 256-byte rows when the image can be mapped that way
+                        if (p.a_map)
+                            tma_load_2d(dst, &map_a, 0, (int)((((int64_t)st * p.wcap + e) * p.entry_bytes) >> 8),
                                         bar_full + 8 * s);
+                        else
+                            bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, bar_full + 8 * s);
+                        if (p.x_map_3d) {
+                            // the NT boxes of X come in with a single 3-D load
+                            tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, bar_full + 8 * s);
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < NT; ++b)
+                                tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow,
+                                            bar_full + 8 * s);
+                        }
+                        if (++s == p.num_stages) { s = 0; ph ^= 1u; }
                     }
-                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
                 }
+                if (!ok) break;
             }
         }
     } else if (warp == 1) {

@@ -57,17 +57,31 @@ spmm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 const int len = p.pair_len[pr];
                 const int32_t *cols = p.pair_col + (int64_t)pr * p.pwcap;
                 const int32_t *src = p.pair_src + (int64_t)pr * p.pwcap * 2 + rank;
+                // list entries are global loads in this thread's serial loop: keep the next four in registers
+                int col_q[4], src_q[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    col_q[u] = u < len ? __ldg(cols + u) : 0;
+                    src_q[u] = u < len ? __ldg(src + 2 * u) : -1;
+                }
                 bool ok = true;
-                for (int e = 0; e < len; ++e) {
-                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t dst = ring + s * p.stage_bytes;
-                    if (leader) mbar_expect_tx(bar_full + 8 * s, 2 * stage_tx);
-                    const int idx = src[2 * e];
-                    const int arow = idx >= 0 ? (int)((((int64_t)st * p.wcap + idx) * p.entry_bytes) >> 8) : p.image_rows;
-                    tma_load_2d_pair(dst, &map_a, 0, arow, leader_full + 8 * s);
-                    tma_load_3d_pair(dst + p.entry_bytes, &map_x, 0, cols[e] * p.bk, ct * 4 + kPairBoxes * (int)rank,
-                                     leader_full + 8 * s);
-                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                for (int e0 = 0; e0 < len && ok; e0 += 4) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int e = e0 + u;
+                        if (e >= len) break;
+                        const int krow = col_q[u] * p.bk;
+                        const int idx = src_q[u];
+                        if (e + 4 < len) { col_q[u] = __ldg(cols + e + 4); src_q[u] = __ldg(src + 2 * (e + 4)); }
+                        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t dst = ring + s * p.stage_bytes;
+                        if (leader) mbar_expect_tx(bar_full + 8 * s, 2 * stage_tx);
+                        const int arow = idx >= 0 ? (int)((((int64_t)st * p.wcap + idx) * p.entry_bytes) >> 8) : p.image_rows;
+                        tma_load_2d_pair(dst, &map_a, 0, arow, leader_full + 8 * s);
+                        tma_load_3d_pair(dst + p.entry_bytes, &map_x, 0, krow, ct * 4 + kPairBoxes * (int)rank,
+                                         leader_full + 8 * s);
+                        if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                    }
                 }
                 if (!ok) break;
             }
