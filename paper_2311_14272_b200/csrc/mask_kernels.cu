@@ -121,12 +121,12 @@ __device__ __forceinline__ unsigned long long fixed_point_score(uint32_t key, in
 
 // Bit i of the result is set iff element i is among the N largest of its group of M
 // (ties to the lower index).  M is 4 or 8; the 8 keys hold two groups or one.
+// For i < j, element i beats element j iff key[i] >= key[j].
 template <int M>
 __device__ __forceinline__ uint32_t top_n_bits(const uint32_t key[8], int n) {
     uint32_t bits = 0u;
 #pragma unroll
     for (int g = 0; g < 8 / M; ++g) {
-        // rank[i] = number of elements that beat element i; for i < j, i beats j iff key[i] >= key[j]
         int rank[M];
 #pragma unroll
         for (int i = 0; i < M; ++i) rank[i] = 0;
@@ -144,6 +144,22 @@ __device__ __forceinline__ uint32_t top_n_bits(const uint32_t key[8], int n) {
     return bits;
 }
 
+// Groups of 4: the six pairwise outcomes index a 64-entry table of keep masks (built per CTA for
+// the layer's n by keep_mask_of_outcomes), which replaces the rank arithmetic.
+__device__ __forceinline__ uint32_t outcomes4(const uint32_t *k) {
+    return (uint32_t)(k[0] >= k[1]) | ((uint32_t)(k[0] >= k[2]) << 1) | ((uint32_t)(k[0] >= k[3]) << 2) |
+           ((uint32_t)(k[1] >= k[2]) << 3) | ((uint32_t)(k[1] >= k[3]) << 4) | ((uint32_t)(k[2] >= k[3]) << 5);
+}
+__device__ __forceinline__ uint32_t keep_mask_of_outcomes(uint32_t o, int n) {
+    const int w01 = o & 1, w02 = (o >> 1) & 1, w03 = (o >> 2) & 1, w12 = (o >> 3) & 1, w13 = (o >> 4) & 1,
+              w23 = (o >> 5) & 1;
+    const int r0 = (1 - w01) + (1 - w02) + (1 - w03);
+    const int r1 = w01 + (1 - w12) + (1 - w13);
+    const int r2 = w02 + w12 + (1 - w23);
+    const int r3 = w03 + w13 + w23;
+    return (uint32_t)(r0 < n) | ((uint32_t)(r1 < n) << 1) | ((uint32_t)(r2 < n) << 2) | ((uint32_t)(r3 < n) << 3);
+}
+
 constexpr int kM1Rows = 32;              // rows per CTA of K-M1 (divides every block height)
 constexpr int kM1RowsPerWarp = kM1Rows / (kM1Threads / 32);
 
@@ -157,6 +173,8 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
                     const uint32_t *__restrict__ max_key, uint32_t *__restrict__ nm_bits,
                     unsigned long long *__restrict__ score) {
     __shared__ unsigned long long s_score[kM1ChunkK / 32 + 2];
+    __shared__ uint8_t s_keep[64];
+    if (M == 4 && threadIdx.x < 64) s_keep[threadIdx.x] = (uint8_t)keep_mask_of_outcomes(threadIdx.x, g.n);
     const int chunk = blockIdx.y;
     const int64_t row0 = (int64_t)blockIdx.x * kM1Rows;
     const int rt = (int)(row0 / g.bm);
@@ -168,6 +186,11 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
 
     const uint32_t mk = *max_key;
     const int e_max = mk ? key_exponent(mk) : 0;
+    // floor(value * 2^(40 - e_max)): when that power of two is an fp32 number, the product is exact
+    // (value <= layer maximum, so it stays below 2^41) and one round-down conversion gives the floor
+    const int scale_exp = kScoreFractionBits - e_max;
+    const bool float_scale = scale_exp >= -126 && scale_exp <= 127;
+    const float scale = float_scale ? __uint_as_float((uint32_t)(127 + scale_exp) << 23) : 0.f;
     const bool in_kp = k0 < g.kp();
     uint32_t key[kM1RowsPerWarp][8];
     if (vec_ok && row0 + kM1Rows <= g.rows && (int64_t)(chunk + 1) * kM1ChunkK <= g.k) {   // interior tile
@@ -186,12 +209,18 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
 #pragma unroll
     for (int i = 0; i < kM1RowsPerWarp; ++i) {
         const int64_t row = row0 + warp * kM1RowsPerWarp + i;
-        const uint32_t bits = top_n_bits<M>(key[i], g.n);
+        uint32_t bits;
+        if constexpr (M == 4)
+            bits = (uint32_t)s_keep[outcomes4(key[i])] | ((uint32_t)s_keep[outcomes4(key[i] + 4)] << 4);
+        else
+            bits = top_n_bits<M>(key[i], g.n);
         const uint32_t counted = g.score_mode == 0 ? bits : 0xFFu;
         if (mk) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                if ((counted >> j) & 1u) acc += fixed_point_score(key[i][j], e_max);
+                if ((counted >> j) & 1u)
+                    acc += float_scale ? __float2ull_rd(__uint_as_float(key[i][j]) * scale)
+                                       : fixed_point_score(key[i][j], e_max);
         }
         uint32_t word = bits << (8 * (lane & 3));
         word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);

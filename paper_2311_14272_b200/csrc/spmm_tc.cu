@@ -301,22 +301,27 @@ build_walk_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int wc
 }
 
 // Union of the walk lists of CTA tiles 2p and 2p+1 (ascending), with each side's entry index.
-__global__ void __launch_bounds__(128)
+// One CTA per pair: bitmap union, then one thread per union entry looks itself up in both lists.
+__global__ void __launch_bounds__(256)
 build_pair_walk_kernel(int nst, int nblk, int wcap, int pwcap, const int32_t *__restrict__ walk_col,
                        const int32_t *__restrict__ walk_len, int32_t *__restrict__ pair_col,
                        int32_t *__restrict__ pair_len, int32_t *__restrict__ pair_src) {
     __shared__ uint32_t s_bits[128];
     __shared__ int s_prefix[129];
+    __shared__ int16_t s_pos[2][4096];               // position of block column jb in each side's list, or -1
     const int p = blockIdx.x;
     const int words = (nblk + 31) / 32;
     for (int i = threadIdx.x; i < words; i += blockDim.x) s_bits[i] = 0u;
+    for (int i = threadIdx.x; i < nblk; i += blockDim.x) { s_pos[0][i] = -1; s_pos[1][i] = -1; }
     __syncthreads();
     for (int side = 0; side < 2; ++side) {
         const int st = 2 * p + side;
         if (st >= nst) continue;
-        for (int i = threadIdx.x; i < walk_len[st]; i += blockDim.x) {
+        const int len = walk_len[st];
+        for (int i = threadIdx.x; i < len; i += blockDim.x) {
             const int jb = walk_col[(int64_t)st * wcap + i];
             atomicOr(&s_bits[jb >> 5], 1u << (jb & 31));
+            s_pos[side][jb] = (int16_t)i;
         }
     }
     __syncthreads();
@@ -326,30 +331,13 @@ build_pair_walk_kernel(int nst, int nblk, int wcap, int pwcap, const int32_t *__
         pair_len[p] = run;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < words; i += blockDim.x) {
-        uint32_t b = s_bits[i];
-        int o = s_prefix[i];
-        while (b) {
-            const int jb = i * 32 + __ffs(b) - 1;
-            b &= b - 1;
-            pair_col[(int64_t)p * pwcap + o] = jb;
-            for (int side = 0; side < 2; ++side) {
-                const int st = 2 * p + side;
-                int found = -1;
-                if (st < nst) {
-                    const int32_t *wc = walk_col + (int64_t)st * wcap;
-                    int lo = 0, hi = walk_len[st] - 1;
-                    while (lo <= hi) {
-                        const int mid = (lo + hi) >> 1;
-                        const int v = wc[mid];
-                        if (v == jb) { found = mid; break; }
-                        if (v < jb) lo = mid + 1; else hi = mid - 1;
-                    }
-                }
-                pair_src[((int64_t)p * pwcap + o) * 2 + side] = found;
-            }
-            ++o;
-        }
+    for (int jb = threadIdx.x; jb < nblk; jb += blockDim.x) {
+        const uint32_t wbits = s_bits[jb >> 5];
+        if (!((wbits >> (jb & 31)) & 1u)) continue;
+        const int o = s_prefix[jb >> 5] + __popc(wbits & ((1u << (jb & 31)) - 1u));
+        pair_col[(int64_t)p * pwcap + o] = jb;
+        pair_src[((int64_t)p * pwcap + o) * 2 + 0] = s_pos[0][jb];
+        pair_src[((int64_t)p * pwcap + o) * 2 + 1] = s_pos[1][jb];
     }
 }
 
@@ -587,7 +575,7 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
     int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
     uint8_t *image = d_exec + L.image_off;
     build_walk_kernel<<<L.nst, 128, 0, st>>>(g, d_blk_col, L.r, L.wcap, walk_col, walk_len);
-    build_pair_walk_kernel<<<L.npairs, 128, 0, st>>>(L.nst, g.nblk, L.wcap, L.pwcap, walk_col, walk_len,
+    build_pair_walk_kernel<<<L.npairs, 256, 0, st>>>(L.nst, g.nblk, L.wcap, L.pwcap, walk_col, walk_len,
                                                       reinterpret_cast<int32_t *>(d_exec + L.pair_col_off),
                                                       reinterpret_cast<int32_t *>(d_exec + L.pair_len_off),
                                                       reinterpret_cast<int32_t *>(d_exec + L.pair_src_off));
