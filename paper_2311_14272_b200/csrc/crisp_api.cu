@@ -176,12 +176,17 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     h->forced_path = -1;
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
+    // 128-row blocks: one kept block is one tensor-core tile, so the encode kernel writes it directly
+    const bool fuse_tiles = h->exec_kind != CRISP_PATH_DIRECT && g.bm == 128;
+    crisp::TcImageLayout L = {};
+    if (h->exec_kind != CRISP_PATH_DIRECT) L = crisp::tc_image_layout(g, h->exec_kind == CRISP_PATH_SPARSE);
     if (e == cudaSuccess)
         e = crisp::launch_encode_canonical(d_w_bf16, ld_w, g, mask->d_blk_col, mask->d_nm_bits,
-                                           h->d_blk_col, h->d_vals, h->d_idx, st);
+                                           h->d_blk_col, h->d_vals, h->d_idx, fuse_tiles ? h->exec_kind : 0,
+                                           fuse_tiles ? h->d_exec + L.image_off : nullptr, L.a_bytes, L.entry_bytes, st);
     if (e == cudaSuccess && h->exec_kind != CRISP_PATH_DIRECT)
         e = crisp::launch_build_image(g, h->exec_kind == CRISP_PATH_SPARSE, h->d_blk_col, h->d_vals, h->d_idx,
-                                      h->d_exec, st);
+                                      h->d_exec, fuse_tiles, st);
     if (e != cudaSuccess) { delete h; return CRISP_CUDA_ERROR; }
     *out = h;
     return CRISP_OK;

@@ -62,6 +62,7 @@ size_t mask_workspace_bytes(const Geometry &g);
 cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geometry &g,
                                     const int32_t *d_mask_blk_col, const uint32_t *d_nm_bits,
                                     int32_t *d_blk_col, uint16_t *d_vals, uint32_t *d_idx,
+                                    int tile_kind, uint8_t *d_image, uint32_t a_bytes, uint32_t entry_bytes,
                                     cudaStream_t st);
 cudaError_t launch_decode(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                           const uint32_t *d_idx, uint16_t *d_w, int64_t ld, cudaStream_t st);
@@ -81,7 +82,7 @@ struct TcImageLayout {
 bool tc_pattern_is_sparse(const Geometry &g);
 TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
 cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
-                               const uint32_t *d_idx, uint8_t *d_exec, cudaStream_t st);
+                               const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, cudaStream_t st);
 bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols);
 cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
                            const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,

@@ -35,12 +35,16 @@ __device__ __forceinline__ void load_group(const uint16_t *__restrict__ w, int64
 // N values of a group land contiguously; values and offsets are staged in shared memory and written
 // out with coalesced 16-byte stores.  Offsets go through a bit stream because a field may straddle
 // two words (3-bit fields for M = 8).
-template <int M>
+// TILE selects what else the CTA emits for 128-row blocks (one kept block = one tensor-core tile):
+// 0 nothing, CRISP_PATH_DENSE the zero-expanded tile, CRISP_PATH_SPARSE the 2:4 compressed tile with
+// its metadata (layouts: see the execution-image kernels of the tensor-core SpMM).
+template <int M, int TILE>
 __global__ void __launch_bounds__(256)
 encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool vec_ok,
                     const int32_t *__restrict__ mask_blk_col, const uint32_t *__restrict__ nm_bits,
                     int32_t *__restrict__ blk_col, uint16_t *__restrict__ vals,
-                    uint32_t *__restrict__ idx) {
+                    uint32_t *__restrict__ idx, uint8_t *__restrict__ image, uint32_t a_bytes,
+                    uint32_t entry_bytes) {
     extern __shared__ uint32_t s_buf[];
     const int blk = blockIdx.x;                       // rt * kkeep + slot
     const int rt = blk / g.kkeep;
@@ -51,7 +55,11 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
     const int val_words = (vpb + 1) / 2;
     uint32_t *s_idx = s_buf;                          // [idx_words]
     uint16_t *s_val = reinterpret_cast<uint16_t *>(s_buf + idx_words);   // [vpb]
+    uint8_t *tile = reinterpret_cast<uint8_t *>(s_buf + idx_words + (vpb + 7) / 8 * 4);   // [entry_bytes], 16-byte aligned
     for (int i = threadIdx.x; i < idx_words; i += blockDim.x) s_idx[i] = 0u;
+    if constexpr (TILE != 0)
+        for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x)
+            reinterpret_cast<uint4 *>(tile)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) blk_col[blk] = jb;
     __syncthreads();
 
@@ -62,6 +70,34 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
         uint16_t v[M];
         load_group<M>(w, ld, g.rows, g.k, row, col0, vec_ok, v);
         uint32_t bits = (nm_bits[row * g.wpr + (col0 >> 5)] >> (col0 & 31)) & ((1u << M) - 1u);
+        if constexpr (TILE == CRISP_PATH_DENSE) {
+#pragma unroll
+            for (int t = 0; t < M; ++t)
+                if ((bits >> t) & 1u) {
+                    const int k = gi * M + t;
+                    *reinterpret_cast<uint16_t *>(tile + (k >> 3) * 2048 + r * 16 + (k & 7) * 2) = v[t];
+                }
+        } else if constexpr (TILE == CRISP_PATH_SPARSE) {
+            uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
+#pragma unroll
+            for (int q = 0; q < M / 4; ++q) {                // aligned 4-groups: at most two kept values each
+                const uint32_t qb = (bits >> (4 * q)) & 0xFu;
+                int p0 = 0, p1 = 1;
+                uint16_t v0 = 0, v1 = 0;
+                if (qb) {
+                    const int first = __ffs(qb) - 1;
+                    const uint32_t rest = qb & (qb - 1);
+                    if (rest) { p0 = first; v0 = v[4 * q + first]; p1 = __ffs(rest) - 1; v1 = v[4 * q + p1]; }
+                    else if (first == 3) { p0 = 0; p1 = 3; v1 = v[4 * q + 3]; }
+                    else { p0 = first; v0 = v[4 * q + first]; p1 = 3; }
+                }
+                const int k0 = gi * M + 4 * q, c0 = k0 >> 1;  // compressed column of the first slot (even)
+                *reinterpret_cast<uint32_t *>(tile + (c0 >> 3) * 2048 + r * 16 + (c0 & 7) * 2) =
+                    (uint32_t)v0 | ((uint32_t)v1 << 16);
+                const int lrow = (r & 7) + 8 * ((k0 >> 4) & 1) + 16 * (r >> 4);
+                atomicOr(&meta[lrow * 4 + (k0 >> 5)], ((uint32_t)p0 | ((uint32_t)p1 << 2)) << ((k0 & 15) + 16 * ((r >> 3) & 1)));
+            }
+        }
         int o = item * g.n;
 #pragma unroll
         for (int t = 0; t < M; ++t) {
@@ -85,6 +121,11 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
     for (int i = threadIdx.x; i < val_words; i += blockDim.x) vout[i] = s_val32[i];
     uint32_t *iout = idx + (int64_t)blk * idx_words;
     for (int i = threadIdx.x; i < idx_words; i += blockDim.x) iout[i] = s_idx[i];
+    if constexpr (TILE != 0) {
+        // with 128-row blocks the walk list of a CTA tile is its row tile's kept list: entry = blk
+        uint4 *out = reinterpret_cast<uint4 *>(image + (int64_t)blk * entry_bytes);
+        for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = reinterpret_cast<uint4 *>(tile)[i];
+    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -117,20 +158,36 @@ decode_block_kernel(Geometry g, const int32_t *__restrict__ blk_col,
 cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geometry &g,
                                     const int32_t *d_mask_blk_col, const uint32_t *d_nm_bits,
                                     int32_t *d_blk_col, uint16_t *d_vals, uint32_t *d_idx,
+                                    int tile_kind, uint8_t *d_image, uint32_t a_bytes, uint32_t entry_bytes,
                                     cudaStream_t st) {
     const int nblocks = g.nrt * g.kkeep;
     if (nblocks == 0) return cudaSuccess;
-    const size_t smem = (size_t)(g.vals_per_block() * g.idx_bits / 32) * sizeof(uint32_t) +
-                        (size_t)(g.vals_per_block() + 2) * sizeof(uint16_t);
+    const size_t vpb = (size_t)g.vals_per_block();
+    size_t smem = (vpb * g.idx_bits / 32) * sizeof(uint32_t) + (vpb + 7) / 8 * 16 + 16;
+    if (tile_kind != 0) smem += entry_bytes;
     // vector loads of a whole group need the group start aligned to its size in every row
     const size_t gbytes = (size_t)g.m * 2;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(d_w) % gbytes == 0) && ((size_t)ld * 2 % gbytes == 0);
-    if (g.m == 4)
-        encode_block_kernel<4><<<nblocks, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits,
-                                                            d_blk_col, d_vals, d_idx);
-    else
-        encode_block_kernel<8><<<nblocks, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits,
-                                                            d_blk_col, d_vals, d_idx);
+#define CRISP_ENCODE_LAUNCH(MV, TV)                                                                          \
+    do {                                                                                                     \
+        auto kern = encode_block_kernel<MV, TV>;                                                             \
+        if (smem > 48 * 1024) {                                                                              \
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            if (e != cudaSuccess) return e;                                                                  \
+        }                                                                                                    \
+        kern<<<nblocks, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits, d_blk_col, d_vals,   \
+                                         d_idx, d_image, a_bytes, entry_bytes);                              \
+    } while (0)
+    if (g.m == 4) {
+        if (tile_kind == CRISP_PATH_SPARSE) CRISP_ENCODE_LAUNCH(4, CRISP_PATH_SPARSE);
+        else if (tile_kind == CRISP_PATH_DENSE) CRISP_ENCODE_LAUNCH(4, CRISP_PATH_DENSE);
+        else CRISP_ENCODE_LAUNCH(4, 0);
+    } else {
+        if (tile_kind == CRISP_PATH_SPARSE) CRISP_ENCODE_LAUNCH(8, CRISP_PATH_SPARSE);
+        else if (tile_kind == CRISP_PATH_DENSE) CRISP_ENCODE_LAUNCH(8, CRISP_PATH_DENSE);
+        else CRISP_ENCODE_LAUNCH(8, 0);
+    }
+#undef CRISP_ENCODE_LAUNCH
     return cudaGetLastError();
 }
 

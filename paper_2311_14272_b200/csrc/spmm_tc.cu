@@ -264,80 +264,61 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
 // --------------------------------------------------------------------- execution image kernels
 
-// Union walk of the r = 128 / bm row tiles that share one CTA tile: ascending block columns.
-// One CTA per CTA tile: mark the kept columns in a shared bitmap, then compact it.
-__global__ void __launch_bounds__(128)
-build_walk_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int wcap,
-                  int32_t *__restrict__ walk_col, int32_t *__restrict__ walk_len) {
-    __shared__ uint32_t s_bits[128];                 // nblk <= 4096
-    __shared__ int s_prefix[129];
-    const int st = blockIdx.x;
-    const int words = (g.nblk + 31) / 32;
-    for (int i = threadIdx.x; i < words; i += blockDim.x) s_bits[i] = 0u;
-    __syncthreads();
-    const int first_rt = st * r;
-    const int n_rt = min(r, g.nrt - first_rt);
-    for (int i = threadIdx.x; i < n_rt * g.kkeep; i += blockDim.x) {
-        const int jb = blk_col[(int64_t)first_rt * g.kkeep + i];
-        atomicOr(&s_bits[jb >> 5], 1u << (jb & 31));
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int i = 0; i < words; ++i) { s_prefix[i] = run; run += __popc(s_bits[i]); }
-        s_prefix[words] = run;
-        walk_len[st] = run;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < words; i += blockDim.x) {
-        uint32_t b = s_bits[i];
-        int o = s_prefix[i];
-        while (b) {
-            const int t = __ffs(b) - 1;
-            b &= b - 1;
-            walk_col[(int64_t)st * wcap + o++] = i * 32 + t;
-        }
-    }
-}
-
-// Union of the walk lists of CTA tiles 2p and 2p+1 (ascending), with each side's entry index.
-// One CTA per pair: bitmap union, then one thread per union entry looks itself up in both lists.
+// Walk lists.  One CTA per pair of adjacent 128-row CTA tiles:
+//   walk of a CTA tile  = ascending union of the kept block columns of its r = 128 / bm row tiles;
+//   walk of the pair    = ascending union of its two CTA tiles' walks, with each side's entry index
+//                         (or -1) for the CTA-pair kernel.
+// Kept columns are marked in shared bitmaps and compacted with a prefix over the bitmap words.
 __global__ void __launch_bounds__(256)
-build_pair_walk_kernel(int nst, int nblk, int wcap, int pwcap, const int32_t *__restrict__ walk_col,
-                       const int32_t *__restrict__ walk_len, int32_t *__restrict__ pair_col,
-                       int32_t *__restrict__ pair_len, int32_t *__restrict__ pair_src) {
-    __shared__ uint32_t s_bits[128];
-    __shared__ int s_prefix[129];
-    __shared__ int16_t s_pos[2][4096];               // position of block column jb in each side's list, or -1
+build_walks_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int nst, int wcap, int pwcap,
+                   int32_t *__restrict__ walk_col, int32_t *__restrict__ walk_len,
+                   int32_t *__restrict__ pair_col, int32_t *__restrict__ pair_len, int32_t *__restrict__ pair_src) {
+    __shared__ uint32_t s_bits[2][128];              // nblk <= 4096
+    __shared__ int s_prefix[3][129];
     const int p = blockIdx.x;
-    const int words = (nblk + 31) / 32;
-    for (int i = threadIdx.x; i < words; i += blockDim.x) s_bits[i] = 0u;
-    for (int i = threadIdx.x; i < nblk; i += blockDim.x) { s_pos[0][i] = -1; s_pos[1][i] = -1; }
+    const int words = (g.nblk + 31) / 32;
+    for (int i = threadIdx.x; i < 2 * 128; i += blockDim.x) s_bits[i >> 7][i & 127] = 0u;
     __syncthreads();
     for (int side = 0; side < 2; ++side) {
         const int st = 2 * p + side;
         if (st >= nst) continue;
-        const int len = walk_len[st];
-        for (int i = threadIdx.x; i < len; i += blockDim.x) {
-            const int jb = walk_col[(int64_t)st * wcap + i];
-            atomicOr(&s_bits[jb >> 5], 1u << (jb & 31));
-            s_pos[side][jb] = (int16_t)i;
+        const int first_rt = st * r;
+        const int n_rt = min(r, g.nrt - first_rt);
+        for (int i = threadIdx.x; i < n_rt * g.kkeep; i += blockDim.x) {
+            const int jb = blk_col[(int64_t)first_rt * g.kkeep + i];
+            atomicOr(&s_bits[side][jb >> 5], 1u << (jb & 31));
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < 3) {                           // prefix of side 0, side 1 and of their union
+        const int which = threadIdx.x;
         int run = 0;
-        for (int i = 0; i < words; ++i) { s_prefix[i] = run; run += __popc(s_bits[i]); }
-        pair_len[p] = run;
+        for (int i = 0; i < words; ++i) {
+            s_prefix[which][i] = run;
+            const uint32_t b = which == 2 ? (s_bits[0][i] | s_bits[1][i]) : s_bits[which][i];
+            run += __popc(b);
+        }
+        if (which == 2) pair_len[p] = run;
+        else if (2 * p + which < nst) walk_len[2 * p + which] = run;
     }
     __syncthreads();
-    for (int jb = threadIdx.x; jb < nblk; jb += blockDim.x) {
-        const uint32_t wbits = s_bits[jb >> 5];
-        if (!((wbits >> (jb & 31)) & 1u)) continue;
-        const int o = s_prefix[jb >> 5] + __popc(wbits & ((1u << (jb & 31)) - 1u));
-        pair_col[(int64_t)p * pwcap + o] = jb;
-        pair_src[((int64_t)p * pwcap + o) * 2 + 0] = s_pos[0][jb];
-        pair_src[((int64_t)p * pwcap + o) * 2 + 1] = s_pos[1][jb];
+    for (int jb = threadIdx.x; jb < g.nblk; jb += blockDim.x) {
+        const int w = jb >> 5;
+        const uint32_t below = (1u << (jb & 31)) - 1u;
+        int pos[2] = {-1, -1};
+        for (int side = 0; side < 2; ++side) {
+            const uint32_t b = s_bits[side][w];
+            if ((b >> (jb & 31)) & 1u) {
+                pos[side] = s_prefix[side][w] + __popc(b & below);
+                walk_col[(int64_t)(2 * p + side) * wcap + pos[side]] = jb;
+            }
+        }
+        if (pos[0] >= 0 || pos[1] >= 0) {
+            const int o = s_prefix[2][w] + __popc((s_bits[0][w] | s_bits[1][w]) & below);
+            pair_col[(int64_t)p * pwcap + o] = jb;
+            pair_src[((int64_t)p * pwcap + o) * 2 + 0] = pos[0];
+            pair_src[((int64_t)p * pwcap + o) * 2 + 1] = pos[1];
+        }
     }
 }
 
@@ -568,17 +549,17 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
 }
 
 cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
-                               const uint32_t *d_idx, uint8_t *d_exec, cudaStream_t st) {
+                               const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, cudaStream_t st) {
     const TcImageLayout L = tc_image_layout(g, sparse);
     if (g.nrt * g.kkeep == 0) return cudaSuccess;
     int32_t *walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
     int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
     uint8_t *image = d_exec + L.image_off;
-    build_walk_kernel<<<L.nst, 128, 0, st>>>(g, d_blk_col, L.r, L.wcap, walk_col, walk_len);
-    build_pair_walk_kernel<<<L.npairs, 256, 0, st>>>(L.nst, g.nblk, L.wcap, L.pwcap, walk_col, walk_len,
-                                                      reinterpret_cast<int32_t *>(d_exec + L.pair_col_off),
-                                                      reinterpret_cast<int32_t *>(d_exec + L.pair_len_off),
-                                                      reinterpret_cast<int32_t *>(d_exec + L.pair_src_off));
+    build_walks_kernel<<<L.npairs, 256, 0, st>>>(g, d_blk_col, L.r, L.nst, L.wcap, L.pwcap, walk_col, walk_len,
+                                                  reinterpret_cast<int32_t *>(d_exec + L.pair_col_off),
+                                                  reinterpret_cast<int32_t *>(d_exec + L.pair_len_off),
+                                                  reinterpret_cast<int32_t *>(d_exec + L.pair_src_off));
+    if (tiles_done) return cudaGetLastError();       // the encode kernel already wrote the weight tiles
     const int grid = L.nst * L.wcap;
     const size_t smem_img = (size_t)L.entry_bytes + (size_t)g.vals_per_block() * 2 + (size_t)(g.vals_per_block() * g.idx_bits / 32) * 4 + 16;
     if (smem_img > 48 * 1024) {      // large blocks with many kept values need the opt-in shared memory size
