@@ -98,20 +98,25 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
                 atomicOr(&meta[lrow * 4 + (k0 >> 5)], ((uint32_t)p0 | ((uint32_t)p1 << 2)) << ((k0 & 15) + 16 * ((r >> 3) & 1)));
             }
         }
+        // values in ascending position; the group's offsets are gathered in a register and merged into
+        // the shared bit stream with one atomic (two if the field straddles a word)
+        constexpr int kIdxBits = M == 4 ? 2 : 3;
         int o = item * g.n;
+        const int bit0 = o * kIdxBits;
+        uint32_t field = 0u;
+        int cnt = 0;
 #pragma unroll
         for (int t = 0; t < M; ++t) {
             if ((bits >> t) & 1u) {
-                s_val[o] = v[t];
-                const int bit = o * g.idx_bits;
-                const uint32_t lo = (uint32_t)t << (bit & 31);
-                if (lo) atomicOr(&s_idx[bit >> 5], lo);
-                if ((bit & 31) + g.idx_bits > 32) {
-                    const uint32_t hi = (uint32_t)t >> (32 - (bit & 31));
-                    if (hi) atomicOr(&s_idx[(bit >> 5) + 1], hi);
-                }
-                ++o;
+                s_val[o + cnt] = v[t];
+                field |= (uint32_t)t << (kIdxBits * cnt);
+                ++cnt;
             }
+        }
+        if (field) {
+            const int sh = bit0 & 31;
+            atomicOr(&s_idx[bit0 >> 5], field << sh);
+            if (sh + kIdxBits * cnt > 32) atomicOr(&s_idx[(bit0 >> 5) + 1], field >> (32 - sh));
         }
     }
     __syncthreads();

@@ -215,12 +215,14 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
         else
             bits = top_n_bits<M>(key[i], g.n);
         const uint32_t counted = g.score_mode == 0 ? bits : 0xFFu;
-        if (mk) {
+        if (float_scale) {                   // uniform over the grid; all-zero layers give scale * 0 = 0
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                if ((counted >> j) & 1u)
-                    acc += float_scale ? __float2ull_rd(__uint_as_float(key[i][j]) * scale)
-                                       : fixed_point_score(key[i][j], e_max);
+                if ((counted >> j) & 1u) acc += __float2ull_rd(__uint_as_float(key[i][j]) * scale);
+        } else if (mk) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if ((counted >> j) & 1u) acc += fixed_point_score(key[i][j], e_max);
         }
         uint32_t word = bits << (8 * (lane & 3));
         word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
