@@ -38,6 +38,48 @@ struct TcParams {
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
 
+constexpr int kWideEpiWarps = 8;                               // two warps per TMEM lane quarter
+constexpr int kWideThreads = 64 + 32 * kWideEpiWarps;          // warp 0 producer, warp 1 MMA issuer, warps 2..9 epilogue
+
+// One epilogue chunk: 32 rows (one per lane) x 128 bytes.  Through the warp's 128B-swizzled staging
+// tile and a TMA store, or, where TMA cannot clip exactly (it clips at 16-byte granularity), with
+// guarded plain stores.
+template <typename OutT>
+__device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap *map_y, uint32_t stg, uint8_t *stg_gen,
+                                            int lane, const uint32_t (&out)[32], int x0, int y0) {
+    constexpr int kOutCols = 128 / (int)sizeof(OutT);
+    if (x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
+        const int row = y0 + lane;
+        if (row < p.rows && x0 < p.ncols) {
+            OutT *dst = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy + x0;
+            const int nvalid = (int)(p.ncols - x0);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                if constexpr (sizeof(OutT) == 2) {
+                    if (2 * i < nvalid) dst[2 * i] = (OutT)(out[i] & 0xFFFFu);
+                    if (2 * i + 1 < nvalid) dst[2 * i + 1] = (OutT)(out[i] >> 16);
+                } else {
+                    if (i < nvalid) dst[i] = __uint_as_float(out[i]);
+                }
+            }
+        }
+        return;
+    }
+    if (lane == 0) bulk_wait_read<0>();          // the previous store has finished reading the staging tile
+    __syncwarp();
+    uint8_t *tile = stg_gen + lane * 128;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)                  // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
+        *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
+            make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        if (x0 < p.ncols && y0 < p.rows) tma_store_2d(map_y, stg, x0, y0);
+        bulk_commit();
+    }
+}
+
 // ----------------------------------------------------------------------------------- kernel
 //
 // Shared memory (1024-byte aligned): num_stages x [weight tile | metadata (sparse) | NT boxes of X]
@@ -47,7 +89,7 @@ struct TcParams {
 // X box layout: TMA SWIZZLE_128B, 64 columns (128 bytes) x bk rows; MN-major operand with 1024 bytes
 // between 8-row K groups and box_bytes between 64-column groups.
 template <int NT, bool kSparse, int kAccStages, typename OutT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kWideThreads, 1)
 spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                const __grid_constant__ CUtensorMap map_a, TcParams p) {
     constexpr int kTileN = NT * kBoxN;
@@ -62,7 +104,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t ring = smem_base;
     const uint32_t staging = ring + p.num_stages * p.stage_bytes;
-    const uint32_t ctrl = staging + kEpiWarps * 2 * kStageTileBytes;
+    const uint32_t ctrl = staging + kWideEpiWarps * kStageTileBytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl - smem_base);
     // barriers: full[s], empty[s] (s < 8), tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = ctrl, bar_empty = ctrl + 64, bar_tfull = ctrl + 128, bar_tempty = ctrl + 144;
@@ -72,7 +114,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < p.num_stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kEpiWarps); }
+        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kWideEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -174,10 +216,16 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
     } else {
         // ------------------------------------------------ epilogue: TMEM -> registers -> smem -> TMA store
-        const int q = warp & 3;                             // TMEM lane quarter this warp may access
-        const uint32_t stg = staging + (uint32_t)(warp - 2) * 2 * kStageTileBytes;
+        // Eight warps.  Warp w may touch TMEM lanes 32*(w%4)..; with an even number of column boxes two
+        // warps share a lane quarter and take half of the columns each: a warp first pulls its whole
+        // share of the accumulator into registers and hands the accumulator back, so that the next
+        // tile's MMAs overlap the conversion and the stores.
+        constexpr bool kSplit = (NT % 2) == 0;
+        constexpr int kWarpCols = kSplit ? kTileN / 2 : kTileN;
+        const int ew = warp - 2, q = warp & 3, half = ew >> 2;
+        const uint32_t stg = staging + (uint32_t)ew * kStageTileBytes;
         uint8_t *stg_gen = smem_gen + (stg - smem_base);
-        uint32_t acc = 0, acc_ph = 0, buf = 0;
+        uint32_t acc = 0, acc_ph = 0;
         for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
             const int st = t % p.nst, ct = t / p.nst;
             int go = 0;                                      // lane 0 waits, the warp follows it
@@ -186,61 +234,55 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             if (!go) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
+            const int y0 = st * kTileM + 32 * q;
+            if constexpr (kSplit) {
+                uint32_t accr[kWarpCols];
+#pragma unroll
+                for (int i = 0; i < kWarpCols / 32; ++i)
+                    tmem_ld32(t_addr + half * kWarpCols + 32 * i, *reinterpret_cast<uint32_t(*)[32]>(&accr[32 * i]));
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);       // accumulator free for the next tile
+#pragma unroll
+                for (int c = 0; c < kWarpCols / kOutCols; ++c) {
+                    uint32_t out[32];
+                    if constexpr (sizeof(OutT) == 2) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            out[i] = pack_bf16(__uint_as_float(accr[c * 64 + 2 * i]), __uint_as_float(accr[c * 64 + 2 * i + 1]));
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) out[i] = accr[c * 32 + i];
+                    }
+                    store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + half * kWarpCols + c * kOutCols, y0);
+                }
+            } else {
+                if (half == 0) {
 #pragma unroll 1
-            for (int c = 0; c < kTileN / kOutCols; ++c) {
-                uint32_t out[32];                            // one 128-byte row per lane
-                if constexpr (sizeof(OutT) == 2) {
-                    uint32_t r0[32], r1[32];
-                    tmem_ld32(t_addr + c * 64, r0);
-                    tmem_ld32(t_addr + c * 64 + 32, r1);
-                    tmem_ld_wait();
+                    for (int c = 0; c < kTileN / kOutCols; ++c) {
+                        uint32_t out[32];
+                        if constexpr (sizeof(OutT) == 2) {
+                            uint32_t r0[32], r1[32];
+                            tmem_ld32(t_addr + c * 64, r0);
+                            tmem_ld32(t_addr + c * 64 + 32, r1);
+                            tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        out[i] = pack_bf16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
-                        out[16 + i] = pack_bf16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
-                    }
-                } else {
-                    tmem_ld32(t_addr + c * 32, out);
-                    tmem_ld_wait();
-                }
-                const int x0 = ct * kTileN + c * kOutCols, y0 = st * kTileM + 32 * q;
-                // TMA clips a store at 16-byte granularity: a chunk that crosses an ncols whose byte
-                // offset is not a multiple of 16 is written with guarded plain stores instead
-                if (x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
-                    const int row = y0 + lane;
-                    if (row < p.rows && x0 < p.ncols) {
-                        OutT *dst = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy + x0;
-                        const int nvalid = (int)(p.ncols - x0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            if constexpr (sizeof(OutT) == 2) {
-                                if (2 * i < nvalid) dst[2 * i] = (OutT)(out[i] & 0xFFFFu);
-                                if (2 * i + 1 < nvalid) dst[2 * i + 1] = (OutT)(out[i] >> 16);
-                            } else {
-                                if (i < nvalid) dst[i] = __uint_as_float(out[i]);
+                            for (int i = 0; i < 16; ++i) {
+                                out[i] = pack_bf16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+                                out[16 + i] = pack_bf16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
                             }
+                        } else {
+                            tmem_ld32(t_addr + c * 32, out);
+                            tmem_ld_wait();
                         }
+                        store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + c * kOutCols, y0);
                     }
-                    continue;
                 }
-                if (lane == 0) bulk_wait_read<1>();          // the staging tile written two stores ago is free
+                tc_fence_before();
                 __syncwarp();
-                uint8_t *tile = stg_gen + buf * kStageTileBytes + lane * 128;
-#pragma unroll
-                for (int j = 0; j < 8; ++j)                  // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
-                    *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
-                        make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    if (x0 < p.ncols && y0 < p.rows) tma_store_2d(&map_y, stg + buf * kStageTileBytes, x0, y0);
-                    bulk_commit();
-                }
-                buf ^= 1u;
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
             if (++acc == kAccStages) { acc = 0; acc_ph ^= 1u; }
         }
         if (lane == 0) bulk_wait_read<0>();
@@ -452,7 +494,7 @@ cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const C
         if (e != cudaSuccess) return e;
         configured = smem;
     }
-    kern<<<grid, kThreads, smem, st>>>(mx, my, ma, p);
+    kern<<<grid, kWideThreads, smem, st>>>(mx, my, ma, p);
     return cudaGetLastError();
 }
 
@@ -613,7 +655,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes;
     p.box_bytes = (uint32_t)(kBoxN * g.bk * 2);
     p.stage_bytes = p.entry_bytes + nt * p.box_bytes;
-    const uint32_t fixed = kEpiWarps * 2 * kStageTileBytes + 256;
+    const uint32_t fixed = kWideEpiWarps * kStageTileBytes + 256;
     uint32_t stages = (kSmemBudget - fixed) / p.stage_bytes;
     if (stages > 8) stages = 8;
     if (stages < 2) return cudaErrorInvalidValue;
