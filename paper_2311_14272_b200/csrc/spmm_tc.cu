@@ -38,6 +38,7 @@ struct TcParams {
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
 
+constexpr uint32_t kWideStageBytes = 2048;                      // epilogue staging tile: 16 rows x 128 bytes
 constexpr int kWideEpiWarps = 8;                               // two warps per TMEM lane quarter
 constexpr int kWideThreads = 64 + 32 * kWideEpiWarps;          // warp 0 producer, warp 1 MMA issuer, warps 2..9 epilogue
 
@@ -65,18 +66,24 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         }
         return;
     }
-    if (lane == 0) bulk_wait_read<0>();          // the previous store has finished reading the staging tile
-    __syncwarp();
-    uint8_t *tile = stg_gen + lane * 128;
+    // the warp's staging tile holds 16 rows: lanes 0..15, then lanes 16..31
 #pragma unroll
-    for (int j = 0; j < 8; ++j)                  // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
-        *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
-            make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
-    fence_async_smem();
-    __syncwarp();
-    if (lane == 0) {
-        if (x0 < p.ncols && y0 < p.rows) tma_store_2d(map_y, stg, x0, y0);
-        bulk_commit();
+    for (int h = 0; h < 2; ++h) {
+        if (lane == 0) bulk_wait_read<0>();      // the previous store has finished reading the staging tile
+        __syncwarp();
+        if ((lane >> 4) == h) {
+            uint8_t *tile = stg_gen + (lane & 15) * 128;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)          // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
+                *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
+                    make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            if (x0 < p.ncols && y0 + 16 * h < p.rows) tma_store_2d(map_y, stg, x0, y0 + 16 * h);
+            bulk_commit();
+        }
     }
 }
 
@@ -99,12 +106,16 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     constexpr int kOutCols = 128 / (int)sizeof(OutT);                // columns of one 128-byte staging row
     constexpr uint32_t kIdesc = make_idesc(kTileN, kSparse);
 
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];     // the kernel has no static shared memory
+    const uint32_t smem_base = smem_u32(smem_raw);
+    uint8_t *smem_gen = smem_raw;
+    if (smem_base & 1023u) {                 // swizzled operand tiles need it; checked, not assumed
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, (int)CRISP_CUDA_ERROR);
+        return;
+    }
     const uint32_t ring = smem_base;
     const uint32_t staging = ring + p.num_stages * p.stage_bytes;
-    const uint32_t ctrl = staging + kWideEpiWarps * kStageTileBytes;
+    const uint32_t ctrl = staging + kWideEpiWarps * kWideStageBytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl - smem_base);
     // barriers: full[s], empty[s] (s < 8), tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = ctrl, bar_empty = ctrl + 64, bar_tfull = ctrl + 128, bar_tempty = ctrl + 144;
@@ -223,7 +234,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         constexpr bool kSplit = (NT % 2) == 0;
         constexpr int kWarpCols = kSplit ? kTileN / 2 : kTileN;
         const int ew = warp - 2, q = warp & 3, half = ew >> 2;
-        const uint32_t stg = staging + (uint32_t)ew * kStageTileBytes;
+        const uint32_t stg = staging + (uint32_t)ew * kWideStageBytes;
         uint8_t *stg_gen = smem_gen + (stg - smem_base);
         uint32_t acc = 0, acc_ph = 0;
         for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
@@ -655,12 +666,12 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes;
     p.box_bytes = (uint32_t)(kBoxN * g.bk * 2);
     p.stage_bytes = p.entry_bytes + nt * p.box_bytes;
-    const uint32_t fixed = kWideEpiWarps * kStageTileBytes + 256;
-    uint32_t stages = (kSmemBudget - fixed) / p.stage_bytes;
+    const uint32_t fixed = kWideEpiWarps * kWideStageBytes + 256;
+    uint32_t stages = (kSmemBudget + 1024 - fixed) / p.stage_bytes;    // the whole 227 KB: the base is 1024-aligned
     if (stages > 8) stages = 8;
     if (stages < 2) return cudaErrorInvalidValue;
     p.num_stages = stages;
-    const size_t smem = (size_t)stages * p.stage_bytes + fixed + 1024;
+    const size_t smem = (size_t)stages * p.stage_bytes + fixed;
 
     CUtensorMap mx, my, ma;
     p.a_map = make_map_image(&ma, p.image, (uint64_t)L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
@@ -672,7 +683,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
         return cudaErrorInvalidValue;
     const bool f32 = y_dtype != 0;
     if (!make_map_2d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, f32 ? 4 : 2, d_y,
-                     (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, 32))
+                     (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, 16))
         return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
 
