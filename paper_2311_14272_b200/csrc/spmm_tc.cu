@@ -653,6 +653,9 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     int nt = (nt_override >= 1 && nt_override <= 4) ? nt_override : 4;
     const int64_t boxes = (ncols + kBoxN - 1) / kBoxN;
     if (boxes < nt) nt = (int)boxes;
+    // small layers are latency-bound: narrower tiles (down to 2 boxes) until at least half of the SMs have one
+    if (nt_override <= 0)
+        while (nt > 2 && (int64_t)L.nst * ((ncols + nt * kBoxN - 1) / (nt * kBoxN)) < sm_count / 2) --nt;
     TcParams p;
     p.image = d_exec + L.image_off;
     p.walk_col = reinterpret_cast<const int32_t *>(d_exec + L.walk_col_off);
