@@ -34,6 +34,8 @@ struct TcParams {
     int nst, wcap, bk, n_col_tiles, num_tiles, rows;
     int64_t ncols;
     uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
+    uint32_t stg_bufs;          // staging tiles per epilogue warp (1, 2 or 4): stores in flight per warp
+    uint32_t walk_cache;        // walk lists are copied into shared memory at kernel start
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
@@ -47,7 +49,7 @@ constexpr int kWideThreads = 64 + 32 * kWideEpiWarps;          // warp 0 produce
 // guarded plain stores.
 template <typename OutT>
 __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap *map_y, uint32_t stg, uint8_t *stg_gen,
-                                            int lane, const uint32_t (&out)[32], int x0, int y0) {
+                                            int lane, const uint32_t (&out)[32], int x0, int y0, uint32_t &slot) {
     constexpr int kOutCols = 128 / (int)sizeof(OutT);
     if (x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
         const int row = y0 + lane;
@@ -66,13 +68,19 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         }
         return;
     }
-    // the warp's staging tile holds 16 rows: lanes 0..15, then lanes 16..31
+    // a staging tile holds 16 rows: lanes 0..15, then lanes 16..31; the warp cycles through stg_bufs tiles
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        if (lane == 0) bulk_wait_read<0>();      // the previous store has finished reading the staging tile
+        if (y0 + 16 * h >= p.rows) break;
+        if (lane == 0) {                         // the store that last used this tile has finished reading it
+            if (p.stg_bufs == 4) bulk_wait_read<3>();
+            else if (p.stg_bufs == 2) bulk_wait_read<1>();
+            else bulk_wait_read<0>();
+        }
         __syncwarp();
+        const uint32_t tile_off = slot * kWideStageBytes;
         if ((lane >> 4) == h) {
-            uint8_t *tile = stg_gen + (lane & 15) * 128;
+            uint8_t *tile = stg_gen + tile_off + (lane & 15) * 128;
 #pragma unroll
             for (int j = 0; j < 8; ++j)          // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
                 *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
@@ -81,16 +89,18 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-            if (x0 < p.ncols && y0 + 16 * h < p.rows) tma_store_2d(map_y, stg, x0, y0 + 16 * h);
+            if (x0 < p.ncols) tma_store_2d(map_y, stg + tile_off, x0, y0 + 16 * h);
             bulk_commit();
         }
+        slot = (slot + 1) & (p.stg_bufs - 1);
     }
 }
 
 // ----------------------------------------------------------------------------------- kernel
 //
 // Shared memory (1024-byte aligned): num_stages x [weight tile | metadata (sparse) | NT boxes of X]
-//                                    | 4 warps x 2 staging tiles | barriers | TMEM base | abort flag
+//                                    | 8 warps x stg_bufs staging tiles | barriers | TMEM base | abort flag
+//                                    | walk lists (optional)
 // Weight tile layout (no swizzle, K-major): [k/8][row][8 elements], i.e. 8x16-byte core matrices are
 // contiguous, 128 bytes between 8-row groups, 2048 bytes between 16-byte K chunks.
 // X box layout: TMA SWIZZLE_128B, 64 columns (128 bytes) x bk rows; MN-major operand with 1024 bytes
@@ -115,12 +125,15 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     const uint32_t ring = smem_base;
     const uint32_t staging = ring + p.num_stages * p.stage_bytes;
-    const uint32_t ctrl = staging + kWideEpiWarps * kWideStageBytes;
+    const uint32_t ctrl = staging + kWideEpiWarps * p.stg_bufs * kWideStageBytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl - smem_base);
     // barriers: full[s], empty[s] (s < 8), tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = ctrl, bar_empty = ctrl + 64, bar_tfull = ctrl + 128, bar_tempty = ctrl + 144;
     volatile uint32_t *tmem_base_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 160);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + 164);
+    // Optional copy of the walk lists ([nst] lengths, then [nst][wcap] block columns): a tile with a short
+    // walk would otherwise spend two dependent global loads per tile in the producer's serial loop.
+    int32_t *s_walk = reinterpret_cast<int32_t *>(ctrl_gen + 256);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -128,7 +141,16 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kWideEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_y);
     }
+    if (p.walk_cache) {
+        for (int i = threadIdx.x; i < p.nst; i += blockDim.x) s_walk[i] = p.walk_len[i];
+        for (int i = threadIdx.x; i < p.nst * p.wcap; i += blockDim.x) s_walk[p.nst + i] = p.walk_col[i];
+    }
+    const int32_t *walk_len = p.walk_cache ? s_walk : p.walk_len;
+    const int32_t *walk_col = p.walk_cache ? s_walk + p.nst : p.walk_col;
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_base_slot)), kTmemCols);
         tmem_relinquish();
@@ -145,14 +167,14 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             uint32_t s = 0, ph = 0;
             for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
                 const int st = t % p.nst, ct = t / p.nst;
-                const int len = p.walk_len[st];
-                const int32_t *cols = p.walk_col + (int64_t)st * p.wcap;
+                const int len = walk_len[st];
+                const int32_t *cols = walk_col + (int64_t)st * p.wcap;
                 const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
                 // The block column of entry e is a global load in this thread's serial loop; left where it
                 // is used it costs one L2 round trip (~0.4 us) per stage.  Keep the next four in registers.
                 int col_q[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) col_q[u] = u < len ? __ldg(cols + u) : 0;
+                for (int u = 0; u < 4; ++u) col_q[u] = u < len ? cols[u] : 0;
                 bool ok = true;
                 for (int e0 = 0; e0 < len && ok; e0 += 4) {
 #pragma unroll
@@ -160,7 +182,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         const int e = e0 + u;
                         if (e >= len) break;
                         const int krow = col_q[u] * p.bk;
-                        if (e + 4 < len) col_q[u] = __ldg(cols + e + 4);
+                        if (e + 4 < len) col_q[u] = cols[e + 4];
                         if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
                         const uint32_t dst = ring + s * p.stage_bytes;
                         mbar_expect_tx(bar_full + 8 * s, tx_bytes);
@@ -191,7 +213,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (lane == 0) {
             uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
             for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
-                const int len = p.walk_len[t % p.nst];
+                const int len = walk_len[t % p.nst];
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1u, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileN;
@@ -234,9 +256,9 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         constexpr bool kSplit = (NT % 2) == 0;
         constexpr int kWarpCols = kSplit ? kTileN / 2 : kTileN;
         const int ew = warp - 2, q = warp & 3, half = ew >> 2;
-        const uint32_t stg = staging + (uint32_t)ew * kWideStageBytes;
+        const uint32_t stg = staging + (uint32_t)ew * p.stg_bufs * kWideStageBytes;
         uint8_t *stg_gen = smem_gen + (stg - smem_base);
-        uint32_t acc = 0, acc_ph = 0;
+        uint32_t acc = 0, acc_ph = 0, slot = 0;
         for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
             const int st = t % p.nst, ct = t / p.nst;
             int go = 0;                                      // lane 0 waits, the warp follows it
@@ -246,7 +268,12 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             tc_fence_after();
             const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
             const int y0 = st * kTileM + 32 * q;
-            if constexpr (kSplit) {
+            if (y0 >= p.rows) {
+                // this lane quarter lies below the last row of W: nothing to drain
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            } else if constexpr (kSplit) {
                 uint32_t accr[kWarpCols];
 #pragma unroll
                 for (int i = 0; i < kWarpCols / 32; ++i)
@@ -266,7 +293,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 32; ++i) out[i] = accr[c * 32 + i];
                     }
-                    store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + half * kWarpCols + c * kOutCols, y0);
+                    store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + half * kWarpCols + c * kOutCols, y0, slot);
                 }
             } else {
                 if (half == 0) {
@@ -287,7 +314,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             tmem_ld32(t_addr + c * 32, out);
                             tmem_ld_wait();
                         }
-                        store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + c * kOutCols, y0);
+                        store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + c * kOutCols, y0, slot);
                     }
                 }
                 tc_fence_before();
@@ -669,12 +696,23 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes;
     p.box_bytes = (uint32_t)(kBoxN * g.bk * 2);
     p.stage_bytes = p.entry_bytes + nt * p.box_bytes;
+    // Shared memory (the whole 227 KB; the base is 1024-aligned): the ring gets as many stages as fit next
+    // to one staging tile per epilogue warp; what is left goes to the walk-list copy and to more staging
+    // tiles.  Short walks are store-heavy and need no deep ring: they give stages up for staging tiles.
+    const uint32_t avail = kSmemBudget + 1024;
     const uint32_t fixed = kWideEpiWarps * kWideStageBytes + 256;
-    uint32_t stages = (kSmemBudget + 1024 - fixed) / p.stage_bytes;    // the whole 227 KB: the base is 1024-aligned
-    if (stages > 8) stages = 8;
+    uint32_t stages = (avail - fixed) / p.stage_bytes;
+    const uint32_t max_stages = L.wcap <= 8 ? (p.stage_bytes <= 24 * 1024 ? 6u : 4u) : 8u;
+    if (stages > max_stages) stages = max_stages;
     if (stages < 2) return cudaErrorInvalidValue;
     p.num_stages = stages;
-    const size_t smem = (size_t)stages * p.stage_bytes + fixed;
+    uint32_t left = avail - fixed - stages * p.stage_bytes;
+    const uint32_t cache_bytes = (uint32_t)align_up((size_t)L.nst * (L.wcap + 1) * sizeof(int32_t), 16);
+    p.walk_cache = cache_bytes <= left ? 1u : 0u;
+    if (p.walk_cache) left -= cache_bytes;
+    p.stg_bufs = left >= 3 * kWideEpiWarps * kWideStageBytes ? 4u : left >= kWideEpiWarps * kWideStageBytes ? 2u : 1u;
+    const size_t smem = (size_t)stages * p.stage_bytes + (size_t)kWideEpiWarps * p.stg_bufs * kWideStageBytes + 256 +
+                        (p.walk_cache ? cache_bytes : 0);
 
     CUtensorMap mx, my, ma;
     p.a_map = make_map_image(&ma, p.image, (uint64_t)L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
