@@ -96,6 +96,59 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
     }
 }
 
+// The MMA issuer's loop, with the number of MMAs per kept block (NM) fixed at compile time: the loop is
+// bound by this one thread's instruction latency, and a straight line of NM MMAs lets the compiler
+// overlap the operand set-up of one MMA with the issue of the previous one.
+// Descriptors of stage 0 are built once; a later stage or K step only moves the start-address field
+// (16-byte units, low word), which cannot carry: shared memory is smaller than 2^18 bytes.  Per K step
+// the weight tile advances by 4096 bytes, X by 32 rows (sparse image, 4096 bytes) or 16 rows (2048).
+struct MmaRoleArgs {
+    uint32_t ring, bar_full, bar_empty, bar_tfull, bar_tempty, tmem_base;
+    const int32_t *walk_len;
+    volatile int *abort_flag;
+};
+template <int kTileN, bool kSparse, int kAccStages, int NM>
+__device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a) {
+    constexpr uint32_t kIdesc = make_idesc(kTileN, kSparse);
+    const uint64_t a_desc0 = make_smem_desc(a.ring, 2048, 128, kLayoutNone);
+    const uint64_t b_desc0 = make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
+    const uint64_t m_desc0 = make_smem_desc(a.ring + p.a_bytes, 128, 128, kLayoutNone);
+    const uint32_t stage_step = p.stage_bytes >> 4, ring_span = p.num_stages * stage_step;
+    uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
+    for (int t = blockIdx.x; t < p.num_tiles && !*a.abort_flag; t += gridDim.x) {
+        const int len = a.walk_len[t % p.nst];
+        if (!mbar_wait(a.bar_tempty + 8 * acc, acc_ph ^ 1u, a.abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = a.tmem_base + acc * kTileN;
+        uint32_t accum = 0;
+        bool ok = true;
+        for (int e = 0; e < len; ++e) {
+            if (!mbar_wait(full, ph, a.abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t ad = a_desc0 + off, bd = b_desc0 + off;
+            if constexpr (kSparse) {
+                const uint32_t meta_tmem = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                tmem_copy_128x128b(meta_tmem, m_desc0 + off);
+#pragma unroll
+                for (int j = 0; j < NM; ++j)
+                    mma_sparse(d_tmem, ad + j * 256, bd + j * 256, kIdesc | (uint32_t)(j & 1), accum | (uint32_t)j,
+                               meta_tmem + (j & ~1));
+                meta_buf ^= 1u;
+            } else {
+#pragma unroll
+                for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * 128, kIdesc, accum | (uint32_t)j);
+            }
+            accum = 1u;
+            mma_commit(empty);                      // stage reusable once these MMAs have read it
+            off += stage_step; full += 8; empty += 8;
+            if (off == ring_span) { off = 0; full = a.bar_full; empty = a.bar_empty; ph ^= 1u; }
+        }
+        if (!ok) break;
+        mma_commit(a.bar_tfull + 8 * acc);          // accumulator complete
+        if (++acc == kAccStages) { acc = 0; acc_ph ^= 1u; }
+    }
+}
+
 // ----------------------------------------------------------------------------------- kernel
 //
 // Shared memory (1024-byte aligned): num_stages x [weight tile | metadata (sparse) | NT boxes of X]
@@ -114,7 +167,6 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     constexpr int kTmemCols = (kAccStages * kTileN + kMetaCols) <= 256 ? 256 : 512;
     static_assert(kAccStages * kTileN + kMetaCols <= 512, "tensor memory is 512 columns");
     constexpr int kOutCols = 128 / (int)sizeof(OutT);                // columns of one 128-byte staging row
-    constexpr uint32_t kIdesc = make_idesc(kTileN, kSparse);
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];     // the kernel has no static shared memory
     const uint32_t smem_base = smem_u32(smem_raw);
@@ -161,48 +213,59 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const uint32_t tmem_base = *tmem_base_slot;
     const uint32_t tx_bytes = p.entry_bytes + NT * p.box_bytes;
 
+    // Both single-thread roles below are bound by their own dependent-instruction latency (one warp per
+    // scheduler, ~5 cycles per dependent instruction), so their per-block loops carry running addresses
+    // (stage base, barrier, image row, descriptors) instead of recomputing them.
     if (warp == 0) {
         // ------------------------------------------------ producer: step 1, kept blocks only
         if (lane == 0) {
-            uint32_t s = 0, ph = 0;
+            constexpr int kAhead = 8;            // block columns held in registers ahead of their use
+            const uint32_t ring_end = ring + p.num_stages * p.stage_bytes;
+            const uint32_t entry_rows = p.entry_bytes >> 8;      // image rows (256 bytes) per walk entry
+            const bool tiled = p.a_map && p.x_map_3d;
+            uint32_t dst = ring, full = bar_full, empty = bar_empty, ph = 0;
             for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
                 const int st = t % p.nst, ct = t / p.nst;
                 const int len = walk_len[st];
                 const int32_t *cols = walk_col + (int64_t)st * p.wcap;
                 const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
-                // The block column of entry e is a global load in this thread's serial loop; left where it
-                // is used it costs one L2 round trip (~0.4 us) per stage.  Keep the next four in registers.
-                int col_q[4];
+                int arow = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
+                // The block column of entry e is a load in this thread's serial loop; left where it is used
+                // it costs a round trip per stage.  Keep the next kAhead in registers.
+                int col_q[kAhead];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) col_q[u] = u < len ? cols[u] : 0;
+                for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
                 bool ok = true;
-                for (int e0 = 0; e0 < len && ok; e0 += 4) {
+                for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < kAhead; ++u) {
                         const int e = e0 + u;
                         if (e >= len) break;
                         const int krow = col_q[u] * p.bk;
-                        if (e + 4 < len) col_q[u] = cols[e + 4];
-                        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-                        const uint32_t dst = ring + s * p.stage_bytes;
-                        mbar_expect_tx(bar_full + 8 * s, tx_bytes);
-                        // untiled bulk copies are served one at a time; tiled loads pipeline, so the weight
-                        // tile is fetched as a box of 256-byte rows when the image can be mapped that way
-                        if (p.a_map)
-                            tma_load_2d(dst, &map_a, 0, (int)((((int64_t)st * p.wcap + e) * p.entry_bytes) >> 8),
-                                        bar_full + 8 * s);
-                        else
-                            bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, bar_full + 8 * s);
-                        if (p.x_map_3d) {
-                            // the NT boxes of X come in with a single 3-D load
-                            tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, bar_full + 8 * s);
+                        if (e + kAhead < len) col_q[u] = cols[e + kAhead];
+                        if (!mbar_wait(empty, ph ^ 1u, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(full, tx_bytes);
+                        if (tiled) {
+                            // tiled loads pipeline (untiled bulk copies are served one at a time): the weight
+                            // tile comes in as a box of 256-byte image rows, the NT boxes of X as one 3-D load
+                            tma_load_2d(dst, &map_a, 0, arow, full);
+                            tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, full);
+                            arow += (int)entry_rows;
                         } else {
+                            if (p.a_map)
+                                tma_load_2d(dst, &map_a, 0, (int)((((int64_t)st * p.wcap + e) * p.entry_bytes) >> 8), full);
+                            else
+                                bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, full);
+                            if (p.x_map_3d) {
+                                tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, full);
+                            } else {
 #pragma unroll
-                            for (int b = 0; b < NT; ++b)
-                                tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow,
-                                            bar_full + 8 * s);
+                                for (int b = 0; b < NT; ++b)
+                                    tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow, full);
+                            }
                         }
-                        if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                        dst += p.stage_bytes; full += 8; empty += 8;
+                        if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
                     }
                 }
                 if (!ok) break;
@@ -211,40 +274,22 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer: steps 2 + 3
         if (lane == 0) {
-            uint32_t s = 0, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
-            for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
-                const int len = walk_len[t % p.nst];
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1u, abort_flag)) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * kTileN;
-                bool ok = true;
-                for (int e = 0; e < len; ++e) {
-                    if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_smem = ring + s * p.stage_bytes;
-                    const uint32_t x_smem = a_smem + p.entry_bytes;
-                    if constexpr (kSparse) {
-                        const uint32_t meta_tmem = tmem_base + kAccStages * kTileN + 4 * meta_buf;
-                        tmem_copy_128x128b(meta_tmem, make_smem_desc(a_smem + p.a_bytes, 128, 128, kLayoutNone));
-                        for (int j = 0; j < p.bk / 32; ++j) {
-                            const uint64_t ad = make_smem_desc(a_smem + j * 4096, 2048, 128, kLayoutNone);
-                            const uint64_t bd = make_smem_desc(x_smem + j * 4096, p.box_bytes, 1024, kLayoutSw128);
-                            mma_sparse(d_tmem, ad, bd, kIdesc | (uint32_t)(j & 1), (e | j) ? 1u : 0u, meta_tmem + (j & ~1));
-                        }
-                        meta_buf ^= 1u;
-                    } else {
-                        for (int j = 0; j < p.bk / 16; ++j) {
-                            const uint64_t ad = make_smem_desc(a_smem + j * 4096, 2048, 128, kLayoutNone);
-                            const uint64_t bd = make_smem_desc(x_smem + j * 2048, p.box_bytes, 1024, kLayoutSw128);
-                            mma_dense(d_tmem, ad, bd, kIdesc, (e | j) ? 1u : 0u);
-                        }
-                    }
-                    mma_commit(bar_empty + 8 * s);          // stage reusable once these MMAs have read it
-                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+            const MmaRoleArgs a{ring, bar_full, bar_empty, bar_tfull, bar_tempty, tmem_base, walk_len, abort_flag};
+            const int nmma = kSparse ? p.bk / 32 : p.bk / 16;        // K = 32 (sparse) or K = 16 steps per block
+            if constexpr (kSparse) {
+                switch (nmma) {
+                    case 1: mma_role<kTileN, true, kAccStages, 1>(p, a); break;
+                    case 2: mma_role<kTileN, true, kAccStages, 2>(p, a); break;
+                    case 3: mma_role<kTileN, true, kAccStages, 3>(p, a); break;
+                    default: mma_role<kTileN, true, kAccStages, 4>(p, a); break;
                 }
-                if (!ok) break;
-                mma_commit(bar_tfull + 8 * acc);            // accumulator complete
-                if (++acc == kAccStages) { acc = 0; acc_ph ^= 1u; }
+            } else {
+                switch (nmma) {
+                    case 2: mma_role<kTileN, false, kAccStages, 2>(p, a); break;
+                    case 4: mma_role<kTileN, false, kAccStages, 4>(p, a); break;
+                    case 6: mma_role<kTileN, false, kAccStages, 6>(p, a); break;
+                    default: mma_role<kTileN, false, kAccStages, 8>(p, a); break;
+                }
             }
         }
     } else {
