@@ -35,6 +35,7 @@ struct TcParams {
     int64_t ncols;
     uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
     uint32_t stg_bufs;          // staging tiles per epilogue warp (1, 2 or 4): stores in flight per warp
+    uint32_t stg_tile_bytes;    // one staging tile: 16 or 32 rows of 128 bytes (= the row count of map_y's box)
     uint32_t walk_cache;        // walk lists are copied into shared memory at kernel start
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
@@ -68,9 +69,10 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         }
         return;
     }
-    // a staging tile holds 16 rows: lanes 0..15, then lanes 16..31; the warp cycles through stg_bufs tiles
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
+    // The warp cycles through stg_bufs staging tiles.  A 32-row tile takes the chunk in one pass and one
+    // store; a 16-row tile (when shared memory is short) takes lanes 0..15, then lanes 16..31.
+    const int passes = p.stg_tile_bytes == 4096 ? 1 : 2;
+    for (int h = 0; h < passes; ++h) {
         if (y0 + 16 * h >= p.rows) break;
         if (lane == 0) {                         // the store that last used this tile has finished reading it
             if (p.stg_bufs == 4) bulk_wait_read<3>();
@@ -78,9 +80,9 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
             else bulk_wait_read<0>();
         }
         __syncwarp();
-        const uint32_t tile_off = slot * kWideStageBytes;
-        if ((lane >> 4) == h) {
-            uint8_t *tile = stg_gen + tile_off + (lane & 15) * 128;
+        const uint32_t tile_off = slot * p.stg_tile_bytes;
+        if (passes == 1 || (lane >> 4) == h) {
+            uint8_t *tile = stg_gen + tile_off + (passes == 1 ? lane : (lane & 15)) * 128;
 #pragma unroll
             for (int j = 0; j < 8; ++j)          // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
                 *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
@@ -152,7 +154,7 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
 // ----------------------------------------------------------------------------------- kernel
 //
 // Shared memory (1024-byte aligned): num_stages x [weight tile | metadata (sparse) | NT boxes of X]
-//                                    | 8 warps x stg_bufs staging tiles | barriers | TMEM base | abort flag
+//                                    | 8 warps x stg_bufs staging tiles (16 or 32 rows) | barriers | TMEM base | abort flag
 //                                    | walk lists (optional)
 // Weight tile layout (no swizzle, K-major): [k/8][row][8 elements], i.e. 8x16-byte core matrices are
 // contiguous, 128 bytes between 8-row groups, 2048 bytes between 16-byte K chunks.
@@ -177,7 +179,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     const uint32_t ring = smem_base;
     const uint32_t staging = ring + p.num_stages * p.stage_bytes;
-    const uint32_t ctrl = staging + kWideEpiWarps * p.stg_bufs * kWideStageBytes;
+    const uint32_t ctrl = staging + kWideEpiWarps * p.stg_bufs * p.stg_tile_bytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl - smem_base);
     // barriers: full[s], empty[s] (s < 8), tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = ctrl, bar_empty = ctrl + 64, bar_tfull = ctrl + 128, bar_tempty = ctrl + 144;
@@ -301,7 +303,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         constexpr bool kSplit = (NT % 2) == 0;
         constexpr int kWarpCols = kSplit ? kTileN / 2 : kTileN;
         const int ew = warp - 2, q = warp & 3, half = ew >> 2;
-        const uint32_t stg = staging + (uint32_t)ew * p.stg_bufs * kWideStageBytes;
+        const uint32_t stg = staging + (uint32_t)ew * p.stg_bufs * p.stg_tile_bytes;
         uint8_t *stg_gen = smem_gen + (stg - smem_base);
         uint32_t acc = 0, acc_ph = 0, slot = 0;
         for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
@@ -747,7 +749,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     const uint32_t avail = kSmemBudget + 1024;
     const uint32_t fixed = kWideEpiWarps * kWideStageBytes + 256;
     uint32_t stages = (avail - fixed) / p.stage_bytes;
-    const uint32_t max_stages = L.wcap <= 8 ? (p.stage_bytes <= 24 * 1024 ? 6u : 4u) : 8u;
+    const uint32_t max_stages = p.stage_bytes <= 24 * 1024 ? (L.wcap <= 8 ? 6u : 7u) : (L.wcap <= 8 ? 4u : 8u);
     if (stages > max_stages) stages = max_stages;
     if (stages < 2) return cudaErrorInvalidValue;
     p.num_stages = stages;
@@ -755,8 +757,12 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     const uint32_t cache_bytes = (uint32_t)align_up((size_t)L.nst * (L.wcap + 1) * sizeof(int32_t), 16);
     p.walk_cache = cache_bytes <= left ? 1u : 0u;
     if (p.walk_cache) left -= cache_bytes;
-    p.stg_bufs = left >= 3 * kWideEpiWarps * kWideStageBytes ? 4u : left >= kWideEpiWarps * kWideStageBytes ? 2u : 1u;
-    const size_t smem = (size_t)stages * p.stage_bytes + (size_t)kWideEpiWarps * p.stg_bufs * kWideStageBytes + 256 +
+    // staging per warp beyond the one 16-row tile already counted: two 32-row tiles, two 16-row tiles, or none
+    const uint32_t unit = kWideEpiWarps * kWideStageBytes;
+    if (left >= 3 * unit) { p.stg_bufs = 2; p.stg_tile_bytes = 2 * kWideStageBytes; }
+    else if (left >= unit) { p.stg_bufs = 2; p.stg_tile_bytes = kWideStageBytes; }
+    else { p.stg_bufs = 1; p.stg_tile_bytes = kWideStageBytes; }
+    const size_t smem = (size_t)stages * p.stage_bytes + (size_t)kWideEpiWarps * p.stg_bufs * p.stg_tile_bytes + 256 +
                         (p.walk_cache ? cache_bytes : 0);
 
     CUtensorMap mx, my, ma;
@@ -769,7 +775,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
         return cudaErrorInvalidValue;
     const bool f32 = y_dtype != 0;
     if (!make_map_2d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, f32 ? 4 : 2, d_y,
-                     (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, 16))
+                     (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, p.stg_tile_bytes / 128))
         return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
 
