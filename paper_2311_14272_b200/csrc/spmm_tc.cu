@@ -42,8 +42,8 @@ struct TcParams {
 };
 
 constexpr uint32_t kWideStageBytes = 2048;                      // epilogue staging tile: 16 rows x 128 bytes
-constexpr int kWideEpiWarps = 8;                               // two warps per TMEM lane quarter
-constexpr int kWideThreads = 64 + 32 * kWideEpiWarps;          // warp 0 producer, warp 1 MMA issuer, warps 2..9 epilogue
+// Epilogue warps: two per TMEM lane quarter, or four where short walks make the epilogue the longest role.
+// Threads: warp 0 producer, warp 1 MMA issuer, then the epilogue warps.
 
 // One epilogue chunk: 32 rows (one per lane) x 128 bytes.  Through the warp's 128B-swizzled staging
 // tile and a TMA store, or, where TMA cannot clip exactly (it clips at 16-byte granularity), with
@@ -160,8 +160,8 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
 // contiguous, 128 bytes between 8-row groups, 2048 bytes between 16-byte K chunks.
 // X box layout: TMA SWIZZLE_128B, 64 columns (128 bytes) x bk rows; MN-major operand with 1024 bytes
 // between 8-row K groups and box_bytes between 64-column groups.
-template <int NT, bool kSparse, int kAccStages, typename OutT>
-__global__ void __launch_bounds__(kWideThreads, 1)
+template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi>
+__global__ void __launch_bounds__(64 + 32 * kEpi, 1)
 spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                const __grid_constant__ CUtensorMap map_a, TcParams p) {
     constexpr int kTileN = NT * kBoxN;
@@ -179,7 +179,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
     const uint32_t ring = smem_base;
     const uint32_t staging = ring + p.num_stages * p.stage_bytes;
-    const uint32_t ctrl = staging + kWideEpiWarps * p.stg_bufs * p.stg_tile_bytes;
+    const uint32_t ctrl = staging + kEpi * p.stg_bufs * p.stg_tile_bytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl - smem_base);
     // barriers: full[s], empty[s] (s < 8), tmem_full[2], tmem_empty[2]
     const uint32_t bar_full = ctrl, bar_empty = ctrl + 64, bar_tfull = ctrl + 128, bar_tempty = ctrl + 144;
@@ -192,7 +192,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < p.num_stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kWideEpiWarps); }
+        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kEpi); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_x);
@@ -296,12 +296,13 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
     } else {
         // ------------------------------------------------ epilogue: TMEM -> registers -> smem -> TMA store
-        // Eight warps.  Warp w may touch TMEM lanes 32*(w%4)..; with an even number of column boxes two
-        // warps share a lane quarter and take half of the columns each: a warp first pulls its whole
-        // share of the accumulator into registers and hands the accumulator back, so that the next
-        // tile's MMAs overlap the conversion and the stores.
-        constexpr bool kSplit = (NT % 2) == 0;
-        constexpr int kWarpCols = kSplit ? kTileN / 2 : kTileN;
+        // Warp w may touch TMEM lanes 32*(w%4)..; the kEpi/4 warps that share a lane quarter split the
+        // tile's columns among them when the shares are whole 64-column boxes: a warp first pulls its
+        // whole share of the accumulator into registers and hands the accumulator back, so that the
+        // next tile's MMAs overlap the conversion and the stores.
+        constexpr int kParts = kEpi / 4;                                  // warps sharing a lane quarter
+        constexpr bool kSplit = (kTileN / kParts) % 64 == 0;
+        constexpr int kWarpCols = kSplit ? kTileN / kParts : kTileN;
         const int ew = warp - 2, q = warp & 3, half = ew >> 2;
         const uint32_t stg = staging + (uint32_t)ew * p.stg_bufs * p.stg_tile_bytes;
         uint8_t *stg_gen = smem_gen + (stg - smem_base);
@@ -569,17 +570,17 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
     for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = s_tile4[i];
 }
 
-template <int NT, bool kSparse, int kAccStages, typename OutT>
+template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi>
 cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const CUtensorMap &ma, const TcParams &p,
                            int grid, size_t smem, cudaStream_t st) {
-    auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT>;
+    auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi>;
     static size_t configured = 0;                       // largest dynamic shared memory opted into so far
     if (smem > configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured = smem;
     }
-    kern<<<grid, kWideThreads, smem, st>>>(mx, my, ma, p);
+    kern<<<grid, 64 + 32 * kEpi, smem, st>>>(mx, my, ma, p);
     return cudaGetLastError();
 }
 
@@ -730,6 +731,11 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     // small layers are latency-bound: narrower tiles (down to 2 boxes) until at least half of the SMs have one
     if (nt_override <= 0)
         while (nt > 2 && (int64_t)L.nst * ((ncols + nt * kBoxN - 1) / (nt * kBoxN)) < sm_count / 2) --nt;
+    // Short walks: the epilogue and the accumulator hand-over are the longest chain.  One warp per 64-column
+    // box and lane quarter; under the sparse image three boxes, so that two accumulators fit beside the
+    // metadata columns and the next tile's MMAs do not wait for the drain.
+    const bool short_walk = L.wcap <= 8 && nt_override <= 0;
+    if (short_walk && L.wcap <= 2 && sparse && nt == 4) nt = 3;
     TcParams p;
     p.image = d_exec + L.image_off;
     p.walk_col = reinterpret_cast<const int32_t *>(d_exec + L.walk_col_off);
@@ -747,7 +753,8 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     // to one staging tile per epilogue warp; what is left goes to the walk-list copy and to more staging
     // tiles.  Short walks are store-heavy and need no deep ring: they give stages up for staging tiles.
     const uint32_t avail = kSmemBudget + 1024;
-    const uint32_t fixed = kWideEpiWarps * kWideStageBytes + 256;
+    const uint32_t epi = short_walk && nt >= 3 ? 4u * (uint32_t)nt : 8u;
+    const uint32_t fixed = epi * kWideStageBytes + 256;
     uint32_t stages = (avail - fixed) / p.stage_bytes;
     const uint32_t max_stages = p.stage_bytes <= 24 * 1024 ? (L.wcap <= 8 ? 6u : 7u) : (L.wcap <= 8 ? 4u : 8u);
     if (stages > max_stages) stages = max_stages;
@@ -758,11 +765,11 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.walk_cache = cache_bytes <= left ? 1u : 0u;
     if (p.walk_cache) left -= cache_bytes;
     // staging per warp beyond the one 16-row tile already counted: two 32-row tiles, two 16-row tiles, or none
-    const uint32_t unit = kWideEpiWarps * kWideStageBytes;
+    const uint32_t unit = epi * kWideStageBytes;
     if (left >= 3 * unit) { p.stg_bufs = 2; p.stg_tile_bytes = 2 * kWideStageBytes; }
     else if (left >= unit) { p.stg_bufs = 2; p.stg_tile_bytes = kWideStageBytes; }
     else { p.stg_bufs = 1; p.stg_tile_bytes = kWideStageBytes; }
-    const size_t smem = (size_t)stages * p.stage_bytes + (size_t)kWideEpiWarps * p.stg_bufs * p.stg_tile_bytes + 256 +
+    const size_t smem = (size_t)stages * p.stage_bytes + (size_t)epi * p.stg_bufs * p.stg_tile_bytes + 256 +
                         (p.walk_cache ? cache_bytes : 0);
 
     CUtensorMap mx, my, ma;
@@ -779,24 +786,26 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
         return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
 
-#define CRISP_TC_LAUNCH(NTV, SP, ACC)                                                                     \
-    (f32 ? launch_variant<NTV, SP, ACC, float>(mx, my, ma, p, grid, smem, st)                                 \
-         : launch_variant<NTV, SP, ACC, uint16_t>(mx, my, ma, p, grid, smem, st))
+#define CRISP_TC_LAUNCH_E(NTV, SP, ACC, EPI)                                                              \
+    (f32 ? launch_variant<NTV, SP, ACC, float, EPI>(mx, my, ma, p, grid, smem, st)                            \
+         : launch_variant<NTV, SP, ACC, uint16_t, EPI>(mx, my, ma, p, grid, smem, st))
+#define CRISP_TC_LAUNCH(NTV, SP, ACC) CRISP_TC_LAUNCH_E(NTV, SP, ACC, 8)
     if (sparse) {
         switch (nt) {
             case 1: return CRISP_TC_LAUNCH(1, true, 2);
             case 2: return CRISP_TC_LAUNCH(2, true, 2);
-            case 3: return CRISP_TC_LAUNCH(3, true, 2);
-            default: return CRISP_TC_LAUNCH(4, true, 1);
+            case 3: return epi == 12 ? CRISP_TC_LAUNCH_E(3, true, 2, 12) : CRISP_TC_LAUNCH(3, true, 2);
+            default: return epi == 16 ? CRISP_TC_LAUNCH_E(4, true, 1, 16) : CRISP_TC_LAUNCH(4, true, 1);
         }
     }
     switch (nt) {
         case 1: return CRISP_TC_LAUNCH(1, false, 2);
         case 2: return CRISP_TC_LAUNCH(2, false, 2);
         case 3: return CRISP_TC_LAUNCH(3, false, 2);
-        default: return CRISP_TC_LAUNCH(4, false, 2);
+        default: return epi == 16 ? CRISP_TC_LAUNCH_E(4, false, 2, 16) : CRISP_TC_LAUNCH(4, false, 2);
     }
 #undef CRISP_TC_LAUNCH
+#undef CRISP_TC_LAUNCH_E
 }
 
 }  // namespace crisp
