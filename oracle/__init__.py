@@ -174,3 +174,34 @@ def spmm_fp64_rows(w_dense, x_bits, sel):
     if rc:
         raise ValueError(f"oracle_spmm_fp64_rows rc={rc}")
     return y
+
+
+def score_scale_exp(saliency: np.ndarray) -> int:
+    """Exponent e of a layer's largest canonical saliency (|s|, NaN -> 0, Inf -> FLT_MAX): one unit of
+    the layer's block scores is worth 2^(e - 40).  0 for an all-zero layer."""
+    s = np.abs(np.nan_to_num(np.asarray(saliency, dtype=np.float32), nan=0.0,
+                             posinf=np.finfo(np.float32).max, neginf=np.finfo(np.float32).max))
+    smax = float(s.max()) if s.size else 0.0
+    return int(np.frexp(smax)[1]) - 1 if smax > 0 else 0      # smax = m * 2^e with m in [0.5, 1)
+
+
+def global_rank(scores, scale_exps, block_elems, prune_fraction: float, min_keep=None) -> np.ndarray:
+    """Algorithm 1, rank-column sums + global order + selection: kept blocks per row tile of every layer.
+
+    scores[l]: uint64 [nrt_l, nblk_l]; scale_exps[l]: int; block_elems[l]: weights per block.
+    """
+    nl = len(scores)
+    arrs = [np.ascontiguousarray(s, dtype=np.uint64) for s in scores]
+    ptrs = (C.POINTER(C.c_uint64) * nl)(*[_p(a, C.c_uint64) for a in arrs])
+    nrt = np.array([a.shape[0] for a in arrs], dtype=np.int32)
+    nblk = np.array([a.shape[1] for a in arrs], dtype=np.int32)
+    se = np.array(scale_exps, dtype=np.int32)
+    be = np.array(block_elems, dtype=np.int64)
+    mk = np.zeros(nl, dtype=np.int32) if min_keep is None else np.array(min_keep, dtype=np.int32)
+    out = np.zeros(nl, dtype=np.int32)
+    rc = lib().oracle_global_rank(C.c_int(nl), ptrs, _p(nrt, C.c_int), _p(nblk, C.c_int), _p(se, C.c_int),
+                                  _p(be, C.c_int64), _p(mk, C.c_int), C.c_double(prune_fraction),
+                                  _p(out, C.c_int32))
+    if rc:
+        raise ValueError(f"oracle_global_rank rc={rc}")
+    return out

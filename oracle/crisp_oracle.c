@@ -14,6 +14,8 @@
  *   - Algorithm 1 sort-per-row + select: the same number of blocks is kept in
  *     every row of the block grid; the lowest-scored are pruned      (Sec. III-C)
  *   - Algorithm 1 "f* = f (.) r": blocks keep their positions        (Sec. III-C)
+ *   - Algorithm 1 rank-column sums c_o, their global order across layers and the
+ *     selection by the sparsity target: how many blocks each layer keeps (Sec. III-C)
  *   - Sec. III-A storage: Blocked-ELLPACK column index per kept block and an
  *     offset in [0, M) per kept value (zero-based, Sec. III-E worked example)
  *   - Sec. III-E three-step sparse product, which equals the masked dense
@@ -354,5 +356,125 @@ int oracle_spmm_fp64_skipzero(const double *w_dense, int rows, int k,
             for (int64_t c = 0; c < ncols; ++c) yr[c] += wv * bf16_to_double(xr[c]);
         }
     }
+    return 0;
+}
+
+/* --------------------------------------------- global rank selection (Algorithm 1) */
+
+/*
+ * Algorithm 1, the steps between the block scores and the pruning itself, over all
+ * layers of a network (Sec. III-C, "Pruning Algorithm"):
+ *   sort    : inside every row of a layer's block grid, order the block scores
+ *             increasingly; S[rt][o] is the o-th smallest score of row tile rt;
+ *   c_o     : add S[rt][o] over the row tiles rt, for every rank position o;
+ *   C_o     : order all c_o of all layers increasingly ("globally across the network");
+ *   select  : prune rank positions from the front of that order until the current
+ *             sparsity target is met.
+ * Pruning rank position o of a layer removes one block from every row tile, so every
+ * row keeps the same number of blocks; since c_o cannot decrease with o, what a
+ * layer loses is always its lowest rank positions, and the result per layer is one
+ * number: kkeep = nblk - (pruned rank positions).
+ *
+ * Readings where the paper is silent:
+ *   - A layer's scores are integers in units of 2^(scale_exp - 40) (the layer's own
+ *     fixed-point scale); rank sums are compared across layers by their real values
+ *     c * 2^scale_exp, exactly.  Ties go to the lower layer index, then the lower o.
+ *   - The target is a number of weights: floor(prune_fraction * total + 0.5), total =
+ *     sum over layers of nrt * nblk * block_elems (whole blocks).  A rank position
+ *     weighs nrt * block_elems.  Positions are pruned in order while the weight
+ *     pruned so far is still below the target (the shortest front that reaches it).
+ *   - The last min_keep rank positions of a layer are never candidates.
+ *
+ * score[l] : [nrt[l]][nblk[l]] block scores of layer l
+ * kkeep_out: [n_layers]
+ */
+typedef unsigned __int128 oracle_u128;
+
+typedef struct {
+    oracle_u128 c;
+    int scale_exp, layer, o;
+    uint64_t weight;
+} oracle_rank_entry;
+
+static int u128_bits(oracle_u128 v)
+{
+    int n = 0;
+    while (v) { ++n; v >>= 1; }
+    return n;
+}
+
+/* sign of a.c * 2^a.scale_exp - b.c * 2^b.scale_exp, then layer, then o */
+static int rank_entry_cmp(const void *pa, const void *pb)
+{
+    const oracle_rank_entry *a = (const oracle_rank_entry *)pa, *b = (const oracle_rank_entry *)pb;
+    int sign = 0;
+    if (a->c == 0 || b->c == 0) {
+        sign = (a->c != 0) - (b->c != 0);
+    } else {
+        const int top_a = u128_bits(a->c) + a->scale_exp, top_b = u128_bits(b->c) + b->scale_exp;
+        if (top_a != top_b) {
+            sign = top_a < top_b ? -1 : 1;
+        } else {
+            /* same leading bit position: bring both to the smaller exponent; the shifted one ends
+             * with exactly as many bits as the other, so nothing is lost */
+            oracle_u128 va = a->c, vb = b->c;
+            if (a->scale_exp > b->scale_exp) va <<= (a->scale_exp - b->scale_exp);
+            else vb <<= (b->scale_exp - a->scale_exp);
+            sign = va < vb ? -1 : (va > vb ? 1 : 0);
+        }
+    }
+    if (sign) return sign;
+    if (a->layer != b->layer) return a->layer < b->layer ? -1 : 1;
+    return a->o < b->o ? -1 : (a->o > b->o ? 1 : 0);
+}
+
+static int u64_cmp(const void *pa, const void *pb)
+{
+    const uint64_t a = *(const uint64_t *)pa, b = *(const uint64_t *)pb;
+    return a < b ? -1 : (a > b ? 1 : 0);
+}
+
+int oracle_global_rank(int n_layers, const uint64_t *const *score, const int *nrt, const int *nblk,
+                       const int *scale_exp, const int64_t *block_elems, const int *min_keep,
+                       double prune_fraction, int32_t *kkeep_out)
+{
+    if (n_layers <= 0 || !score || !nrt || !nblk || !scale_exp || !block_elems || !min_keep || !kkeep_out) return -1;
+    if (!(prune_fraction >= 0.0 && prune_fraction <= 1.0)) return -1;
+    int64_t n_entries = 0;
+    double total = 0.0;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!score[l] || nrt[l] <= 0 || nblk[l] <= 0 || block_elems[l] <= 0 || min_keep[l] < 0) return -1;
+        n_entries += nblk[l];
+        total += (double)nrt[l] * (double)nblk[l] * (double)block_elems[l];
+    }
+    const uint64_t target = (uint64_t)floor(prune_fraction * total + 0.5);
+    oracle_rank_entry *entry = (oracle_rank_entry *)malloc(sizeof(oracle_rank_entry) * (size_t)n_entries);
+    if (!entry) return -2;
+    int64_t n = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        uint64_t *row = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)nblk[l]);
+        oracle_u128 *c = (oracle_u128 *)calloc((size_t)nblk[l], sizeof(oracle_u128));
+        if (!row || !c) { free(row); free(c); free(entry); return -2; }
+        for (int rt = 0; rt < nrt[l]; ++rt) {
+            memcpy(row, score[l] + (int64_t)rt * nblk[l], sizeof(uint64_t) * (size_t)nblk[l]);
+            qsort(row, (size_t)nblk[l], sizeof(uint64_t), u64_cmp);          /* sort per row, increasing */
+            for (int o = 0; o < nblk[l]; ++o) c[o] += row[o];                /* c_o: sum down the column */
+        }
+        const int candidates = nblk[l] - min_keep[l];
+        for (int o = 0; o < candidates; ++o) {
+            entry[n].c = c[o]; entry[n].scale_exp = scale_exp[l]; entry[n].layer = l; entry[n].o = o;
+            entry[n].weight = (uint64_t)nrt[l] * (uint64_t)block_elems[l];
+            ++n;
+        }
+        kkeep_out[l] = nblk[l];
+        free(row); free(c);
+    }
+    qsort(entry, (size_t)n, sizeof(oracle_rank_entry), rank_entry_cmp);      /* C_o: global order */
+    uint64_t pruned = 0;
+    for (int64_t i = 0; i < n && pruned < target; ++i) {                     /* select by the target */
+        pruned += entry[i].weight;
+        kkeep_out[entry[i].layer] -= 1;
+    }
+    free(entry);
     return 0;
 }
