@@ -230,6 +230,56 @@ def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=12):
     return out
 
 
+def measure_global_rank(torch, B, dev, with_oracle, iters=12):
+    """Global rank selection (Algorithm 1: per-row sort, rank-column sums, global order, selection by the
+    sparsity target) over the VGG-16 and MobileNetV2 stand-in networks: device time of crisp_global_rank
+    on the block scores that crisp_build_mask left on the device, and the oracle's time for the same step."""
+    out = []
+    stream = torch.cuda.current_stream()
+    for name, cfg in (("vgg16", wl.config3()), ("mobilenetv2", wl.config4())):
+        layers, sal = [], []
+        for l in cfg:
+            s = wl.make_saliency(l, wl.make_weight(l))
+            L = B.HybridLayer(l.rows, l.k, l.n, l.m, l.block_rows, l.block_k, 1.0, device=dev)
+            L.build_mask(torch.from_numpy(s).to(dev))
+            layers.append(L); sal.append(s)
+        arr = B.make_rank_layers([L.rank_layer(1) for L in layers])
+        ws = torch.empty(B.crisp_global_rank_sizes(arr), dtype=torch.uint8, device=dev)
+        kk = torch.zeros(len(layers), dtype=torch.int32, device=dev)
+        ts = []
+        for i in range(3 + iters):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            B.crisp_global_rank(arr, 0.6, ws, kk)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        rec = {"network": name, "layers": len(layers), "rank_positions": int(sum(L.nblk - 1 for L in layers)),
+               "block_scores": int(sum(L.nrt * L.nblk for L in layers)), "prune_fraction": 0.6,
+               "global_rank_us": float(np.mean(ts)) * 1e3, "launches": 3,
+               "kkeep": kk.cpu().numpy().tolist()}
+        if with_oracle:
+            import oracle
+            import time
+            scores = []
+            for L in layers:
+                sc_ptr, _ = B.crisp_mask_scores(L.desc, L.workspace)
+                off = sc_ptr - L.workspace.data_ptr()
+                scores.append(L.workspace[off: off + 8 * L.nrt * L.nblk].view(torch.int64).cpu().numpy()
+                              .view(np.uint64).reshape(L.nrt, L.nblk))
+            exps = [oracle.score_scale_exp(s) for s in sal]
+            elems = [L.desc.block_rows * L.desc.block_k for L in layers]
+            t0 = time.perf_counter()
+            want = oracle.global_rank(scores, exps, elems, 0.6, min_keep=[1] * len(layers))
+            rec["oracle_us"] = (time.perf_counter() - t0) * 1e6
+            rec["matches_oracle"] = bool(np.array_equal(want, np.array(rec["kkeep"])))
+        for L in layers:
+            L.close()
+        out.append(rec)
+    return out
+
+
 def recorded_traffic(workload, kernel):
     """DRAM bytes per launch from the committed ncu capture, or None when the kernel source has
     changed since the counters were taken."""
@@ -416,6 +466,7 @@ def run_ours(args, layer, rank, world):
 
     if rank == 0 and world == 1 and not args.no_cells and args.workload.startswith("sweep_"):
         out["cells"] = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
+        out["global_rank"] = measure_global_rank(torch, B, dev, not args.no_cpu_baseline)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)

@@ -112,7 +112,8 @@ CRISP_API crisp_status_t crisp_mask_sizes(const crisp_layer_desc_t *desc, size_t
  *               NaN counts as 0, +-Inf as FLT_MAX.
  *   d_mask_buf  out, mask_bytes; holds blk_col[nrt, kkeep] (int32, ascending per row tile)
  *               and nm_bits[nrt*block_rows, nblk*block_k/32] (uint32, bit k%32 of word k/32).
- *   d_workspace scratch, workspace_bytes; contents undefined afterwards.
+ *   d_workspace scratch, workspace_bytes; afterwards it holds the layer's block scores (see
+ *               crisp_mask_scores) until it is reused.
  *   out         receives a mask object that refers to d_mask_buf (not to d_saliency or
  *               d_workspace).  Free it with crisp_mask_destroy.
  * Steps: per group of m elements keep the n largest |s| (ties: lower k); block score =
@@ -152,6 +153,52 @@ CRISP_API crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s,
 CRISP_API crisp_status_t crisp_build_mask_static(const float *d_saliency, int64_t ld_s,
                                                  const crisp_layer_desc_t *desc, void *d_mask_buf,
                                                  void *stream, crisp_mask_t *out);
+
+/*
+ * Global rank selection across the layers of a network: Algorithm 1 of the paper between the
+ * block scores and the pruning itself (Sec. III-C, "Pruning Algorithm": sort the block scores
+ * inside every row of the block grid, add the o-th smallest score of every row into the
+ * rank-column sum c_o, order all c_o of all layers increasingly, and prune from the front of
+ * that order until the current sparsity target is met).  Pruning rank position o of a layer
+ * removes one block from every row tile, so every row keeps the same number of blocks; the
+ * result per layer is that number, kkeep, which crisp_build_mask then takes as
+ * keep_ratio = kkeep / nblk.
+ *
+ * Inputs are the block scores crisp_build_mask leaves in its workspace.  After that call (with
+ * any keep ratio) and until the workspace is reused, the workspace holds the bits of the
+ * layer's largest |s| (uint32, byte 0; it fixes the unit of the scores, 2^(e_max - 40)) and the
+ * [nrt, nblk] uint64 scores (byte 256); crisp_mask_scores returns the two addresses.
+ *
+ * Readings where the paper is silent:
+ *   - rank sums of different layers are compared by their real values c * 2^(e_max - 40),
+ *     exactly (128-bit integers); ties go to the lower layer index, then the lower o;
+ *   - the target is a number of weights, floor(prune_fraction * total + 0.5) with total = sum
+ *     over layers of nrt * nblk * block_elems; a rank position weighs nrt * block_elems;
+ *     positions are pruned in order while the weight pruned so far is below the target.
+ *     With Algorithm 1's overall sparsity kappa_p and N:M inside kept blocks,
+ *     prune_fraction = 1 - (1 - kappa_p) * M / N;
+ *   - the last min_keep rank positions of a layer are never pruned (0 lets a layer vanish).
+ *
+ * layers (host array) is read before the call returns.  d_workspace: crisp_global_rank_sizes
+ * bytes, 256-byte aligned, scratch.  d_kkeep: device, int32 [n_layers], written on `stream`.
+ * nblk <= 4096 per layer (CRISP_UNSUPPORTED beyond).  Nothing is allocated.
+ */
+typedef struct {
+    const unsigned long long *d_scores;  /* device, [nrt, nblk] block scores                      */
+    const uint32_t *d_max_key;           /* device, bits of the layer's largest |s|               */
+    int32_t nrt, nblk;                   /* row tiles, k-blocks per row tile                      */
+    int64_t block_elems;                 /* weights per block: block_rows * block_k               */
+    int32_t min_keep;                    /* blocks per row tile that are never pruned             */
+    int32_t reserved;                    /* 0                                                     */
+} crisp_rank_layer_t;
+
+CRISP_API crisp_status_t crisp_mask_scores(const crisp_layer_desc_t *desc, const void *d_workspace,
+                                           const unsigned long long **d_scores, const uint32_t **d_max_key);
+CRISP_API crisp_status_t crisp_global_rank_sizes(int32_t n_layers, const crisp_rank_layer_t *layers,
+                                                 size_t *workspace_bytes);
+CRISP_API crisp_status_t crisp_global_rank(int32_t n_layers, const crisp_rank_layer_t *layers,
+                                           double prune_fraction, void *d_workspace, int32_t *d_kkeep,
+                                           void *stream);
 
 /* Copy the mask to host: h_blk_col [nrt*kkeep] int32, h_nm_bits [nrt*block_rows *
  * nblk*block_k/32] uint32.  Either may be NULL.  Synchronises `stream`. */

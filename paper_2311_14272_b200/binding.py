@@ -24,6 +24,11 @@ class LayerDesc(C.Structure):
                 ("score_mode", C.c_int32)]
 
 
+class RankLayer(C.Structure):
+    _fields_ = [("d_scores", C.c_void_p), ("d_max_key", C.c_void_p), ("nrt", C.c_int32), ("nblk", C.c_int32),
+                ("block_elems", C.c_int64), ("min_keep", C.c_int32), ("reserved", C.c_int32)]
+
+
 class BytesModel(C.Structure):
     _fields_ = [("nnz", C.c_int64), ("vals_bytes", C.c_int64), ("idx_bytes", C.c_int64),
                 ("blk_col_bytes", C.c_int64), ("x_bytes", C.c_int64), ("y_bytes", C.c_int64),
@@ -72,6 +77,9 @@ def load(path: Optional[str] = None):
         "crisp_set_path": [vp, i32],
         "crisp_device_status": [vp, vp, P(i32)],
         "crisp_bytes_model": [vp, i64, i32, P(BytesModel)],
+        "crisp_mask_scores": [P(LayerDesc), vp, P(vp), P(vp)],
+        "crisp_global_rank_sizes": [i32, P(RankLayer), P(sz)],
+        "crisp_global_rank": [i32, P(RankLayer), C.c_double, vp, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -135,6 +143,34 @@ def crisp_mask_sizes(desc: LayerDesc):
     a, b = C.c_size_t(), C.c_size_t()
     _check(load().crisp_mask_sizes(C.byref(desc), C.byref(a), C.byref(b)), "crisp_mask_sizes")
     return a.value, b.value
+
+
+def crisp_mask_scores(desc: LayerDesc, d_workspace):
+    """-> (address of the [nrt, nblk] uint64 block scores, address of the max-key word) inside a workspace
+    that crisp_build_mask has filled."""
+    a, b = C.c_void_p(), C.c_void_p()
+    _check(load().crisp_mask_scores(C.byref(desc), _ptr(d_workspace), C.byref(a), C.byref(b)), "crisp_mask_scores")
+    return a.value, b.value
+
+
+def make_rank_layers(layers):
+    """layers: iterable of (d_scores, d_max_key, nrt, nblk, block_elems, min_keep) -> ctypes array."""
+    layers = list(layers)
+    arr = (RankLayer * len(layers))()
+    for i, (sc, mk, nrt, nblk, be, keep) in enumerate(layers):
+        arr[i] = RankLayer(_ptr(sc), _ptr(mk), nrt, nblk, be, keep, 0)
+    return arr
+
+
+def crisp_global_rank_sizes(rank_layers) -> int:
+    out = C.c_size_t()
+    _check(load().crisp_global_rank_sizes(len(rank_layers), rank_layers, C.byref(out)), "crisp_global_rank_sizes")
+    return out.value
+
+
+def crisp_global_rank(rank_layers, prune_fraction: float, d_workspace, d_kkeep, stream=None):
+    _check(load().crisp_global_rank(len(rank_layers), rank_layers, float(prune_fraction), _ptr(d_workspace),
+                                    _ptr(d_kkeep), _stream(stream)), "crisp_global_rank")
 
 
 def crisp_build_mask(d_saliency, ld_s: int, desc: LayerDesc, d_mask_buf, d_workspace, stream=None) -> int:
@@ -253,6 +289,21 @@ class HybridLayer:
         assert saliency.is_cuda and saliency.dtype == self.torch.float32 and saliency.stride(1) == 1
         crisp_mask_destroy(self.mask)
         self.mask = crisp_build_mask(saliency, saliency.stride(0), self.desc, self.mask_buf, self.workspace, stream)
+        return self
+
+    def rank_layer(self, min_keep=0):
+        """This layer's entry for crisp_global_rank (valid after build_mask, until the workspace is reused)."""
+        sc, mk = crisp_mask_scores(self.desc, self.workspace)
+        return (sc, mk, self.nrt, self.nblk, self.desc.block_rows * self.desc.block_k, min_keep)
+
+    def set_kkeep(self, kkeep: int):
+        """Keep ratio that makes the next build_mask keep exactly `kkeep` blocks per row tile."""
+        self.desc.keep_ratio = float(kkeep) / float(self.nblk)
+        self.nblk, self.kkeep = crisp_keep_count(self.desc)
+        assert self.kkeep == kkeep
+        mask_bytes, ws_bytes = crisp_mask_sizes(self.desc)
+        if self.mask_buf.numel() < mask_bytes:
+            self.mask_buf = self.torch.empty(mask_bytes, dtype=self.torch.uint8, device=self.device)
         return self
 
     def export_mask(self, stream=None):

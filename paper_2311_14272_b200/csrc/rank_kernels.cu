@@ -1,0 +1,251 @@
+// Global rank selection across layers (Algorithm 1 of the paper, between the block scores and the
+// pruning itself; Sec. III-C "Pruning Algorithm"):
+//   K-R1  per layer: sort every row of the block-score grid increasingly and add the o-th smallest
+//         score of every row tile into the rank-column sum c_o (128-bit: sums can pass 2^64);
+//   K-R2  global order of all c_o of all layers by their real value c * 2^e (e = the layer's score
+//         scale), ties to the lower layer, then the lower rank position; a rank position is pruned
+//         while the weight of everything before it in that order is still below the target;
+//   K-R3  kkeep = nblk - pruned rank positions, per layer.
+// The order is not materialised: every candidate adds up the weight of the candidates that precede
+// it (all pairs, tiled through shared memory).  The lists are small (one entry per rank position per
+// layer: hundreds to a few thousand for the networks of Sec. IV), so the quadratic pass costs
+// microseconds, is exact, and has no data-dependent control flow.
+#include <cmath>
+#include <vector>
+
+#include "crisp_internal.h"
+
+namespace crisp {
+namespace {
+
+constexpr int kRankThreads = 256;
+constexpr int kRankMaxBlocks = 4096;                 // k-blocks per row tile (one shared-memory row)
+
+struct RankLayer {                                   // device copy of one crisp_rank_layer_t
+    const unsigned long long *scores;
+    const uint32_t *max_key;
+    long long block_elems;
+    int nrt, nblk, candidates, entry_off;
+};
+
+struct RankEntry {
+    unsigned long long lo, hi;                       // c_o
+    unsigned long long weight;                       // weights removed by pruning this rank position
+    int exp, layer, o, pad;
+};
+
+// Exponent of a positive finite float given by its bits (ilogb), denormals included; 0 for zero.
+__device__ __forceinline__ int float_bits_exponent(uint32_t key) {
+    if (!key) return 0;
+    const int e = (int)(key >> 23);
+    return e ? e - 127 : (31 - __clz(key)) - 149;
+}
+
+__device__ __forceinline__ int bit_length(unsigned long long lo, unsigned long long hi) {
+    return hi ? 128 - __clzll(hi) : (lo ? 64 - __clzll(lo) : 0);
+}
+
+// sign of a.c * 2^a.exp - b.c * 2^b.exp, exactly
+__device__ __forceinline__ int compare_values(const RankEntry &a, const RankEntry &b) {
+    const bool az = (a.lo | a.hi) == 0, bz = (b.lo | b.hi) == 0;
+    if (az || bz) return (int)bz - (int)az;
+    const int top_a = bit_length(a.lo, a.hi) + a.exp, top_b = bit_length(b.lo, b.hi) + b.exp;
+    if (top_a != top_b) return top_a < top_b ? -1 : 1;
+    // equal leading-bit position: shift the operand with the larger exponent left by the difference;
+    // it then has exactly as many bits as the other one, so nothing leaves the 128 bits
+    unsigned long long alo = a.lo, ahi = a.hi, blo = b.lo, bhi = b.hi;
+    const int d = a.exp - b.exp;
+    const int sh = d >= 0 ? d : -d;
+    if (sh) {
+        unsigned long long &lo = d > 0 ? alo : blo, &hi = d > 0 ? ahi : bhi;
+        if (sh >= 64) { hi = lo << (sh - 64); lo = 0; }
+        else { hi = (hi << sh) | (lo >> (64 - sh)); lo <<= sh; }
+    }
+    if (ahi != bhi) return ahi < bhi ? -1 : 1;
+    if (alo != blo) return alo < blo ? -1 : 1;
+    return 0;
+}
+
+// K-R1.  One CTA per layer; rows one after the other (bitonic sort in shared memory), thread t owns
+// rank positions t, t + 256, ...
+__global__ void __launch_bounds__(kRankThreads)
+rank_columns_kernel(const RankLayer *__restrict__ layers, RankEntry *__restrict__ entries) {
+    __shared__ unsigned long long s_row[kRankMaxBlocks];
+    const RankLayer L = layers[blockIdx.x];
+    int padded = 1;
+    while (padded < L.nblk) padded <<= 1;
+    constexpr int kPerThread = kRankMaxBlocks / kRankThreads;
+    unsigned long long lo[kPerThread], hi[kPerThread];
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) lo[i] = hi[i] = 0;
+    for (int rt = 0; rt < L.nrt; ++rt) {
+        const unsigned long long *row = L.scores + (long long)rt * L.nblk;
+        for (int i = threadIdx.x; i < padded; i += kRankThreads) s_row[i] = i < L.nblk ? row[i] : ~0ull;
+        __syncthreads();
+        for (int k = 2; k <= padded; k <<= 1)
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int i = threadIdx.x; i < padded; i += kRankThreads) {
+                    const int partner = i ^ j;
+                    if (partner > i) {
+                        const unsigned long long a = s_row[i], b = s_row[partner];
+                        const bool up = (i & k) == 0;
+                        if ((a > b) == up) { s_row[i] = b; s_row[partner] = a; }
+                    }
+                }
+                __syncthreads();
+            }
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            const int o = threadIdx.x + i * kRankThreads;
+            if (o < L.nblk) {
+                const unsigned long long v = s_row[o];
+                lo[i] += v;
+                hi[i] += lo[i] < v;                  // carry
+            }
+        }
+        __syncthreads();
+    }
+    const int e = float_bits_exponent(*L.max_key);
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+        const int o = threadIdx.x + i * kRankThreads;
+        if (o < L.candidates) {
+            RankEntry out;
+            out.lo = lo[i]; out.hi = hi[i];
+            out.weight = (unsigned long long)L.nrt * (unsigned long long)L.block_elems;
+            out.exp = e; out.layer = blockIdx.x; out.o = o; out.pad = 0;
+            entries[L.entry_off + o] = out;
+        }
+    }
+}
+
+// K-R2.  Thread i: weight of the candidates that precede candidate i in the global order.
+__global__ void __launch_bounds__(kRankThreads)
+global_select_kernel(const RankEntry *__restrict__ entries, int n, unsigned long long target,
+                     int32_t *__restrict__ pruned) {
+    __shared__ RankEntry s_tile[kRankThreads];
+    const int i = blockIdx.x * kRankThreads + threadIdx.x;
+    RankEntry mine;
+    if (i < n) mine = entries[i];
+    unsigned long long before = 0;
+    for (int base = 0; base < n; base += kRankThreads) {
+        if (base + (int)threadIdx.x < n) s_tile[threadIdx.x] = entries[base + threadIdx.x];
+        __syncthreads();
+        const int cnt = min(kRankThreads, n - base);
+        if (i < n)
+            for (int j = 0; j < cnt; ++j) {
+                const RankEntry &other = s_tile[j];
+                int c = compare_values(other, mine);
+                if (c == 0) c = other.layer != mine.layer ? (other.layer < mine.layer ? -1 : 1)
+                                                          : (other.o < mine.o ? -1 : (other.o > mine.o ? 1 : 0));
+                if (c < 0) before += other.weight;
+            }
+        __syncthreads();
+    }
+    if (i < n && before < target) atomicAdd(&pruned[mine.layer], 1);
+}
+
+// K-R3.
+__global__ void kept_count_kernel(const RankLayer *__restrict__ layers, const int32_t *__restrict__ pruned,
+                                  int n_layers, int32_t *__restrict__ kkeep) {
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l < n_layers) kkeep[l] = layers[l].nblk - pruned[l];
+}
+
+struct RankLayout {
+    size_t table_off, pruned_off, entries_off, total;
+    long long n_entries;
+};
+
+crisp_status_t rank_layout(int32_t n_layers, const crisp_rank_layer_t *layers, RankLayout *out) {
+    if (n_layers <= 0 || !layers) return CRISP_INVALID_ARG;
+    long long n = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const crisp_rank_layer_t &L = layers[l];
+        if (L.nrt <= 0 || L.nblk <= 0 || L.block_elems <= 0) return CRISP_BAD_SHAPE;
+        if (L.min_keep < 0 || L.min_keep > L.nblk) return CRISP_INVALID_ARG;
+        if (L.nblk > kRankMaxBlocks) return CRISP_UNSUPPORTED;
+        n += L.nblk - L.min_keep;
+    }
+    if (n > 0x7FFFFFFF) return CRISP_UNSUPPORTED;
+    out->n_entries = n;
+    out->table_off = 0;
+    out->pruned_off = align_up((size_t)n_layers * sizeof(RankLayer));
+    out->entries_off = out->pruned_off + align_up((size_t)n_layers * sizeof(int32_t));
+    out->total = out->entries_off + align_up((size_t)(n > 0 ? n : 1) * sizeof(RankEntry));
+    return CRISP_OK;
+}
+
+}  // namespace
+}  // namespace crisp
+
+using crisp::RankEntry;
+using crisp::RankLayer;
+using crisp::RankLayout;
+
+extern "C" {
+
+CRISP_API crisp_status_t crisp_global_rank_sizes(int32_t n_layers, const crisp_rank_layer_t *layers,
+                                                 size_t *workspace_bytes) {
+    if (!workspace_bytes) return CRISP_INVALID_ARG;
+    RankLayout lay;
+    crisp_status_t s = crisp::rank_layout(n_layers, layers, &lay);
+    if (s != CRISP_OK) return s;
+    *workspace_bytes = lay.total;
+    return CRISP_OK;
+}
+
+CRISP_API crisp_status_t crisp_global_rank(int32_t n_layers, const crisp_rank_layer_t *layers, double prune_fraction,
+                                           void *d_workspace, int32_t *d_kkeep, void *stream) {
+    RankLayout lay;
+    crisp_status_t s = crisp::rank_layout(n_layers, layers, &lay);
+    if (s != CRISP_OK) return s;
+    if (!d_workspace || !d_kkeep || reinterpret_cast<uintptr_t>(d_workspace) % crisp::kAlign) return CRISP_INVALID_ARG;
+    if (!(prune_fraction >= 0.0 && prune_fraction <= 1.0)) return CRISP_INVALID_ARG;
+    std::vector<RankLayer> table((size_t)n_layers);
+    double total = 0.0;
+    int off = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const crisp_rank_layer_t &L = layers[l];
+        if (!L.d_scores || !L.d_max_key) return CRISP_INVALID_ARG;
+        table[l].scores = L.d_scores;
+        table[l].max_key = L.d_max_key;
+        table[l].block_elems = L.block_elems;
+        table[l].nrt = L.nrt; table[l].nblk = L.nblk;
+        table[l].candidates = L.nblk - L.min_keep;
+        table[l].entry_off = off;
+        off += table[l].candidates;
+        total += (double)L.nrt * (double)L.nblk * (double)L.block_elems;
+    }
+    const unsigned long long target = (unsigned long long)floor(prune_fraction * total + 0.5);
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = reinterpret_cast<uint8_t *>(d_workspace);
+    RankLayer *d_table = reinterpret_cast<RankLayer *>(ws + lay.table_off);
+    int32_t *d_pruned = reinterpret_cast<int32_t *>(ws + lay.pruned_off);
+    RankEntry *d_entries = reinterpret_cast<RankEntry *>(ws + lay.entries_off);
+    // the table is read from pageable host memory: the call returns once it has been staged
+    if (cudaMemcpyAsync(d_table, table.data(), table.size() * sizeof(RankLayer), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return CRISP_CUDA_ERROR;
+    if (cudaMemsetAsync(d_pruned, 0, (size_t)n_layers * sizeof(int32_t), st) != cudaSuccess) return CRISP_CUDA_ERROR;
+    crisp::rank_columns_kernel<<<n_layers, crisp::kRankThreads, 0, st>>>(d_table, d_entries);
+    const int n = (int)lay.n_entries;
+    if (n > 0)
+        crisp::global_select_kernel<<<(n + crisp::kRankThreads - 1) / crisp::kRankThreads, crisp::kRankThreads, 0, st>>>(
+            d_entries, n, target, d_pruned);
+    crisp::kept_count_kernel<<<(n_layers + 255) / 256, 256, 0, st>>>(d_table, d_pruned, n_layers, d_kkeep);
+    return cudaGetLastError() == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
+}
+
+CRISP_API crisp_status_t crisp_mask_scores(const crisp_layer_desc_t *desc, const void *d_workspace,
+                                           const unsigned long long **d_scores, const uint32_t **d_max_key) {
+    if (!desc || !d_workspace || !d_scores || !d_max_key) return CRISP_INVALID_ARG;
+    size_t mask_bytes = 0, ws_bytes = 0;
+    crisp_status_t s = crisp_mask_sizes(desc, &mask_bytes, &ws_bytes);
+    if (s != CRISP_OK) return s;
+    const uint8_t *ws = reinterpret_cast<const uint8_t *>(d_workspace);
+    *d_max_key = reinterpret_cast<const uint32_t *>(ws);
+    *d_scores = reinterpret_cast<const unsigned long long *>(ws + crisp::kAlign);
+    return CRISP_OK;
+}
+
+}  // extern "C"
