@@ -6,10 +6,11 @@
 //         scale), ties to the lower layer, then the lower rank position; a rank position is pruned
 //         while the weight of everything before it in that order is still below the target;
 //   K-R3  kkeep = nblk - pruned rank positions, per layer.
-// The order is not materialised: every candidate adds up the weight of the candidates that precede
-// it (all pairs, tiled through shared memory).  The lists are small (one entry per rank position per
+// The order is not materialised: for every candidate one warp adds up the weight of the candidates that
+// precede it (all pairs, tiled through shared memory).  The lists are small (one entry per rank position per
 // layer: hundreds to a few thousand for the networks of Sec. IV), so the quadratic pass costs
 // microseconds, is exact, and has no data-dependent control flow.
+#include <climits>
 #include <cmath>
 #include <vector>
 
@@ -28,10 +29,14 @@ struct RankLayer {                                   // device copy of one crisp
     int nrt, nblk, candidates, entry_off;
 };
 
+// One candidate rank position.  Its value c * 2^e is stored normalised, so that the global order is a
+// plain lexicographic comparison: `top` = position of the leading bit of the real value (bit length of
+// c plus e; INT_MIN for c = 0) and the 128-bit c shifted left until its leading bit is bit 127.  Two
+// non-zero values with the same `top` compare like their left-aligned digits; nothing is rounded.
 struct RankEntry {
-    unsigned long long lo, hi;                       // c_o
+    unsigned long long mhi, mlo;
     unsigned long long weight;                       // weights removed by pruning this rank position
-    int exp, layer, o, pad;
+    int top, layer, o, pad;
 };
 
 // Exponent of a positive finite float given by its bits (ilogb), denormals included; 0 for zero.
@@ -41,59 +46,111 @@ __device__ __forceinline__ int float_bits_exponent(uint32_t key) {
     return e ? e - 127 : (31 - __clz(key)) - 149;
 }
 
-__device__ __forceinline__ int bit_length(unsigned long long lo, unsigned long long hi) {
-    return hi ? 128 - __clzll(hi) : (lo ? 64 - __clzll(lo) : 0);
+__device__ __forceinline__ RankEntry make_entry(unsigned long long lo, unsigned long long hi, int e, int layer, int o,
+                                                unsigned long long weight) {
+    RankEntry out;
+    out.weight = weight; out.layer = layer; out.o = o; out.pad = 0;
+    if ((lo | hi) == 0) { out.top = INT_MIN; out.mhi = out.mlo = 0; return out; }
+    const int bits = hi ? 128 - __clzll(hi) : 64 - __clzll(lo);
+    const int sh = 128 - bits;                       // 0..127
+    if (sh >= 64) { out.mhi = lo << (sh - 64); out.mlo = 0; }
+    else if (sh) { out.mhi = (hi << sh) | (lo >> (64 - sh)); out.mlo = lo << sh; }
+    else { out.mhi = hi; out.mlo = lo; }
+    out.top = bits + e;
+    return out;
 }
 
-// sign of a.c * 2^a.exp - b.c * 2^b.exp, exactly
-__device__ __forceinline__ int compare_values(const RankEntry &a, const RankEntry &b) {
-    const bool az = (a.lo | a.hi) == 0, bz = (b.lo | b.hi) == 0;
-    if (az || bz) return (int)bz - (int)az;
-    const int top_a = bit_length(a.lo, a.hi) + a.exp, top_b = bit_length(b.lo, b.hi) + b.exp;
-    if (top_a != top_b) return top_a < top_b ? -1 : 1;
-    // equal leading-bit position: shift the operand with the larger exponent left by the difference;
-    // it then has exactly as many bits as the other one, so nothing leaves the 128 bits
-    unsigned long long alo = a.lo, ahi = a.hi, blo = b.lo, bhi = b.hi;
-    const int d = a.exp - b.exp;
-    const int sh = d >= 0 ? d : -d;
-    if (sh) {
-        unsigned long long &lo = d > 0 ? alo : blo, &hi = d > 0 ? ahi : bhi;
-        if (sh >= 64) { hi = lo << (sh - 64); lo = 0; }
-        else { hi = (hi << sh) | (lo >> (64 - sh)); lo <<= sh; }
-    }
-    if (ahi != bhi) return ahi < bhi ? -1 : 1;
-    if (alo != blo) return alo < blo ? -1 : 1;
-    return 0;
+// a strictly before b in the global order: value, then layer, then rank position (branch-free, so that
+// the loads of consecutive comparisons overlap)
+__device__ __forceinline__ bool entry_before(const RankEntry &a, const RankEntry &b) {
+    const bool by_pos = (a.layer < b.layer) | ((a.layer == b.layer) & (a.o < b.o));
+    const bool by_lo = (a.mlo < b.mlo) | ((a.mlo == b.mlo) & by_pos);
+    const bool by_hi = (a.mhi < b.mhi) | ((a.mhi == b.mhi) & by_lo);
+    return (a.top < b.top) | ((a.top == b.top) & by_hi);
 }
 
-// K-R1.  One CTA per layer; rows one after the other (bitonic sort in shared memory), thread t owns
-// rank positions t, t + 256, ...
+// Increasing bitonic sort of `padded` (a power of two) values in shared memory by `nthreads` threads that
+// call it together; `sync` separates the exchange steps (the warp or the whole CTA).
+template <typename Sync>
+__device__ __forceinline__ void bitonic_sort(unsigned long long *v, int padded, int tid, int nthreads, Sync sync) {
+    for (int k = 2; k <= padded; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < padded; i += nthreads) {
+                const int partner = i ^ j;
+                if (partner > i) {
+                    const unsigned long long a = v[i], b = v[partner];
+                    if ((a > b) == ((i & k) == 0)) { v[i] = b; v[partner] = a; }
+                }
+            }
+            sync();
+        }
+}
+
+constexpr int kWarpRowMax = 512;                     // rows up to this (padded) length are sorted by one warp each
+
+// K-R1.  One CTA per layer.  Rows of up to 512 blocks: each of the 8 warps sorts its own rows in its
+// slice of shared memory and keeps its partial rank sums in registers (lane t owns positions t, t + 32,
+// ...); the warps' sums are then added up in shared memory.  Longer rows: the whole CTA sorts one row
+// at a time (thread t owns positions t, t + 256, ...).
 __global__ void __launch_bounds__(kRankThreads)
 rank_columns_kernel(const RankLayer *__restrict__ layers, RankEntry *__restrict__ entries) {
     __shared__ unsigned long long s_row[kRankMaxBlocks];
+    __shared__ unsigned long long s_lo[kWarpRowMax], s_hi[kWarpRowMax];
     const RankLayer L = layers[blockIdx.x];
     int padded = 1;
     while (padded < L.nblk) padded <<= 1;
-    constexpr int kPerThread = kRankMaxBlocks / kRankThreads;
+    const int e = float_bits_exponent(*L.max_key);
+    const unsigned long long weight = (unsigned long long)L.nrt * (unsigned long long)L.block_elems;
+    constexpr int kPerThread = kRankMaxBlocks / kRankThreads;        // = kWarpRowMax / 32
     unsigned long long lo[kPerThread], hi[kPerThread];
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) lo[i] = hi[i] = 0;
+
+    if (padded <= kWarpRowMax) {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        unsigned long long *mine = s_row + warp * kWarpRowMax;
+        for (int rt = warp; rt < L.nrt; rt += kRankThreads / 32) {
+            const unsigned long long *row = L.scores + (long long)rt * L.nblk;
+            for (int i = lane; i < padded; i += 32) mine[i] = i < L.nblk ? row[i] : ~0ull;
+            __syncwarp();
+            bitonic_sort(mine, padded, lane, 32, [] { __syncwarp(); });
+#pragma unroll
+            for (int i = 0; i < kPerThread; ++i) {
+                const int o = lane + i * 32;
+                if (o < L.nblk) {
+                    const unsigned long long v = mine[o];
+                    lo[i] += v;
+                    hi[i] += lo[i] < v;              // carry
+                }
+            }
+            __syncwarp();
+        }
+        for (int i = threadIdx.x; i < kWarpRowMax; i += kRankThreads) s_lo[i] = s_hi[i] = 0;
+        __syncthreads();
+        for (int w = 0; w < kRankThreads / 32; ++w) {
+            if (warp == w) {
+#pragma unroll
+                for (int i = 0; i < kPerThread; ++i) {
+                    const int o = lane + i * 32;
+                    if (o < L.nblk) {
+                        const unsigned long long before = s_lo[o];
+                        s_lo[o] = before + lo[i];
+                        s_hi[o] += hi[i] + (s_lo[o] < before);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        for (int o = threadIdx.x; o < L.candidates; o += kRankThreads)
+            entries[L.entry_off + o] = make_entry(s_lo[o], s_hi[o], e, blockIdx.x, o, weight);
+        return;
+    }
+
     for (int rt = 0; rt < L.nrt; ++rt) {
         const unsigned long long *row = L.scores + (long long)rt * L.nblk;
         for (int i = threadIdx.x; i < padded; i += kRankThreads) s_row[i] = i < L.nblk ? row[i] : ~0ull;
         __syncthreads();
-        for (int k = 2; k <= padded; k <<= 1)
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                for (int i = threadIdx.x; i < padded; i += kRankThreads) {
-                    const int partner = i ^ j;
-                    if (partner > i) {
-                        const unsigned long long a = s_row[i], b = s_row[partner];
-                        const bool up = (i & k) == 0;
-                        if ((a > b) == up) { s_row[i] = b; s_row[partner] = a; }
-                    }
-                }
-                __syncthreads();
-            }
+        bitonic_sort(s_row, padded, threadIdx.x, kRankThreads, [] { __syncthreads(); });
 #pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
             const int o = threadIdx.x + i * kRankThreads;
@@ -105,44 +162,40 @@ rank_columns_kernel(const RankLayer *__restrict__ layers, RankEntry *__restrict_
         }
         __syncthreads();
     }
-    const int e = float_bits_exponent(*L.max_key);
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
         const int o = threadIdx.x + i * kRankThreads;
-        if (o < L.candidates) {
-            RankEntry out;
-            out.lo = lo[i]; out.hi = hi[i];
-            out.weight = (unsigned long long)L.nrt * (unsigned long long)L.block_elems;
-            out.exp = e; out.layer = blockIdx.x; out.o = o; out.pad = 0;
-            entries[L.entry_off + o] = out;
-        }
+        if (o < L.candidates) entries[L.entry_off + o] = make_entry(lo[i], hi[i], e, blockIdx.x, o, weight);
     }
 }
 
-// K-R2.  Thread i: weight of the candidates that precede candidate i in the global order.
+// K-R2.  One warp per candidate i: the lanes share out the other candidates (tiled through shared memory),
+// each adds up the weight of those that precede i in the global order, and a shuffle reduction gives the
+// weight pruned before i.
 __global__ void __launch_bounds__(kRankThreads)
 global_select_kernel(const RankEntry *__restrict__ entries, int n, unsigned long long target,
                      int32_t *__restrict__ pruned) {
     __shared__ RankEntry s_tile[kRankThreads];
-    const int i = blockIdx.x * kRankThreads + threadIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (kRankThreads / 32) + warp;
     RankEntry mine;
+    mine.top = 0; mine.mhi = mine.mlo = 0; mine.layer = mine.o = 0;
     if (i < n) mine = entries[i];
     unsigned long long before = 0;
     for (int base = 0; base < n; base += kRankThreads) {
         if (base + (int)threadIdx.x < n) s_tile[threadIdx.x] = entries[base + threadIdx.x];
         __syncthreads();
         const int cnt = min(kRankThreads, n - base);
-        if (i < n)
-            for (int j = 0; j < cnt; ++j) {
-                const RankEntry &other = s_tile[j];
-                int c = compare_values(other, mine);
-                if (c == 0) c = other.layer != mine.layer ? (other.layer < mine.layer ? -1 : 1)
-                                                          : (other.o < mine.o ? -1 : (other.o > mine.o ? 1 : 0));
-                if (c < 0) before += other.weight;
-            }
+#pragma unroll 4
+        for (int j = lane; j < cnt; j += 32) {
+            const RankEntry other = s_tile[j];
+            before += entry_before(other, mine) ? other.weight : 0ull;
+        }
         __syncthreads();
     }
-    if (i < n && before < target) atomicAdd(&pruned[mine.layer], 1);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, d);
+    if (i < n && lane == 0 && before < target) atomicAdd(&pruned[mine.layer], 1);
 }
 
 // K-R3.
@@ -230,7 +283,7 @@ CRISP_API crisp_status_t crisp_global_rank(int32_t n_layers, const crisp_rank_la
     crisp::rank_columns_kernel<<<n_layers, crisp::kRankThreads, 0, st>>>(d_table, d_entries);
     const int n = (int)lay.n_entries;
     if (n > 0)
-        crisp::global_select_kernel<<<(n + crisp::kRankThreads - 1) / crisp::kRankThreads, crisp::kRankThreads, 0, st>>>(
+        crisp::global_select_kernel<<<(n + crisp::kRankThreads / 32 - 1) / (crisp::kRankThreads / 32), crisp::kRankThreads, 0, st>>>(
             d_entries, n, target, d_pruned);
     crisp::kept_count_kernel<<<(n_layers + 255) / 256, 256, 0, st>>>(d_table, d_pruned, n_layers, d_kkeep);
     return cudaGetLastError() == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
