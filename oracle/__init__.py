@@ -205,3 +205,21 @@ def global_rank(scores, scale_exps, block_elems, prune_fraction: float, min_keep
     if rc:
         raise ValueError(f"oracle_global_rank rc={rc}")
     return out
+
+
+def conv_fp64(w_dense: np.ndarray, kh: int, kw: int, act_bits: np.ndarray, pad: int) -> np.ndarray:
+    """Convolution by its definition (stride 1, zero padding): w_dense fp64 [S, kh*kw*R] with the reduction
+    ordered (kernel row, kernel column, channel); act_bits bf16 patterns [B, H, W, R] -> fp64 [S, B*Ho*Wo]."""
+    wd = np.ascontiguousarray(w_dense, dtype=np.float64)
+    a = np.ascontiguousarray(act_bits, dtype=np.uint16)
+    b, h, w, r = a.shape
+    s = wd.shape[0]
+    assert wd.shape[1] == kh * kw * r
+    ho, wo = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    y = np.zeros((s, b * ho * wo), dtype=np.float64)
+    rc = lib().oracle_conv_fp64(_p(wd, C.c_double), C.c_int(s), C.c_int(kh), C.c_int(kw), C.c_int(r),
+                                _p(a, C.c_uint16), C.c_int(b), C.c_int(h), C.c_int(w), C.c_int(pad),
+                                _p(y, C.c_double))
+    if rc:
+        raise ValueError(f"oracle_conv_fp64 rc={rc}")
+    return y

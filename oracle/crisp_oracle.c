@@ -19,7 +19,8 @@
  *   - Sec. III-A storage: Blocked-ELLPACK column index per kept block and an
  *     offset in [0, M) per kept value (zero-based, Sec. III-E worked example)
  *   - Sec. III-E three-step sparse product, which equals the masked dense
- *     product; the oracle is that definition: decode, then an fp64 triple loop.
+ *     product; the oracle is that definition: decode, then an fp64 triple loop;
+ *     for a convolution layer, the definition of the convolution (no lowering).
  *
  * Readings where the paper is silent (mirrored in the design notes):
  *   rows of W are output channels and groups/blocks run along the reduction
@@ -476,5 +477,46 @@ int oracle_global_rank(int n_layers, const uint64_t *const *score, const int *nr
         kkeep_out[entry[i].layer] -= 1;
     }
     free(entry);
+    return 0;
+}
+
+/* ------------------------------------------------ convolution as implicit GEMM */
+
+/*
+ * The same product for a convolution layer (Sec. III, Notation: a K x K x R x S filter bank is the
+ * matrix W with S rows, one per output channel, and K*K*R reduction elements; the paper runs the
+ * hybrid pattern on that matrix).  The oracle is the definition of the convolution, with the
+ * reduction index of W ordered (kernel row, kernel column, input channel), channel fastest:
+ *
+ *   Y[s, b, y, x] = sum over (i, j, r) of Wd[s, (i*kw + j)*R + r] * A[b, y + i - pad, x + j - pad, r]
+ *
+ * stride 1, zero padding `pad` on every side, A in NHWC order [batch, height, width, R] as bf16 bit
+ * patterns, Y as [S, batch*ho*wo] with ho = height + 2*pad - kh + 1 (wo likewise), fp64 accumulation
+ * in ascending (i, j, r) order.  w_dense is the decoded masked weight, [S, kh*kw*R] in fp64.
+ */
+int oracle_conv_fp64(const double *w_dense, int s_out, int kh, int kw, int r_in,
+                     const uint16_t *act, int batch, int height, int width, int pad, double *y)
+{
+    if (!w_dense || !act || !y || s_out <= 0 || kh <= 0 || kw <= 0 || r_in <= 0) return -1;
+    if (batch <= 0 || height <= 0 || width <= 0 || pad < 0) return -1;
+    const int ho = height + 2 * pad - kh + 1, wo = width + 2 * pad - kw + 1;
+    if (ho <= 0 || wo <= 0) return -1;
+    const int64_t k = (int64_t)kh * kw * r_in, npix = (int64_t)batch * ho * wo;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int s = 0; s < s_out; ++s)
+        for (int b = 0; b < batch; ++b)
+            for (int oy = 0; oy < ho; ++oy)
+                for (int ox = 0; ox < wo; ++ox) {
+                    double acc = 0.0;
+                    for (int i = 0; i < kh; ++i)
+                        for (int j = 0; j < kw; ++j) {
+                            const int iy = oy + i - pad, ix = ox + j - pad;
+                            if (iy < 0 || iy >= height || ix < 0 || ix >= width) continue;   /* zero padding */
+                            const uint16_t *a = act + (((int64_t)b * height + iy) * width + ix) * r_in;
+                            const double *wr = w_dense + (int64_t)s * k + ((int64_t)i * kw + j) * r_in;
+                            for (int r = 0; r < r_in; ++r) acc += wr[r] * bf16_to_double(a[r]);
+                        }
+                    y[(int64_t)s * npix + ((int64_t)b * ho + oy) * wo + ox] = acc;
+                }
     return 0;
 }

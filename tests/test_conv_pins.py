@@ -1,0 +1,64 @@
+"""Pins for the oracle's convolution (the layer product of Sec. III with W viewed as an S x (K*K*R)
+matrix): against an independently lowered im2col + matrix product, and on kernels whose result is
+known without computing anything."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2311_14272_b200 import workloads as wl
+
+
+def bf16(a):
+    return wl.f32_to_bf16_bits(np.asarray(a, dtype=np.float32))
+
+
+def im2col(act, kh, kw, pad):
+    """[B,H,W,R] -> [kh*kw*R, B*Ho*Wo], reduction ordered (i, j, r), by numpy slicing of a padded copy."""
+    b, h, w, r = act.shape
+    ho, wo = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    p = np.zeros((b, h + 2 * pad, w + 2 * pad, r), dtype=act.dtype)
+    p[:, pad:pad + h, pad:pad + w, :] = act
+    cols = np.empty((kh, kw, r, b, ho, wo), dtype=act.dtype)
+    for i in range(kh):
+        for j in range(kw):
+            cols[i, j] = np.transpose(p[:, i:i + ho, j:j + wo, :], (3, 0, 1, 2))
+    return cols.reshape(kh * kw * r, b * ho * wo)
+
+
+@pytest.mark.parametrize("b,h,w,r,s,kh,kw,pad", [(2, 5, 7, 3, 4, 3, 3, 1), (1, 6, 4, 8, 5, 3, 3, 0),
+                                                 (3, 4, 4, 2, 3, 1, 1, 0), (2, 5, 5, 4, 2, 5, 3, 2)])
+def test_equals_im2col_product(b, h, w, r, s, kh, kw, pad):
+    rng = np.random.default_rng(b * 100 + h)
+    act = bf16(rng.standard_normal((b, h, w, r)))
+    wd = rng.standard_normal((s, kh * kw * r))
+    x = wl.bf16_bits_to_f32(im2col(act, kh, kw, pad)).astype(np.float64)
+    got = oracle.conv_fp64(wd, kh, kw, act, pad)
+    np.testing.assert_allclose(got, wd @ x, rtol=1e-12, atol=1e-12)
+    if kh == kw == 1:
+        # a 1x1 convolution is the plain product with the activation matrix
+        np.testing.assert_allclose(got, oracle.spmm_fp64(wd, act.reshape(-1, r).T.copy()), rtol=0, atol=1e-12)
+
+
+def test_one_hot_taps_shift_the_image():
+    rng = np.random.default_rng(5)
+    b, h, w, r = 2, 6, 5, 3
+    act = bf16(rng.standard_normal((b, h, w, r)))
+    a = wl.bf16_bits_to_f32(act).astype(np.float64)
+    for (i, j, ch) in [(1, 1, 0), (0, 0, 2), (2, 1, 1), (1, 2, 0)]:
+        wd = np.zeros((1, 9 * r))
+        wd[0, (i * 3 + j) * r + ch] = 1.0
+        got = oracle.conv_fp64(wd, 3, 3, act, 1).reshape(b, h, w)
+        want = np.zeros((b, h, w))
+        for y in range(h):
+            for x in range(w):
+                iy, ix = y + i - 1, x + j - 1
+                if 0 <= iy < h and 0 <= ix < w:
+                    want[:, y, x] = a[:, iy, ix, ch]
+        assert np.array_equal(got, want)       # picks: exact, including the zero border
+
+
+def test_all_ones_kernel_counts_the_window():
+    act = bf16(np.ones((1, 4, 4, 2)))
+    got = oracle.conv_fp64(np.ones((1, 18)), 3, 3, act, 1).reshape(4, 4)
+    inside = np.array([[4, 6, 6, 4], [6, 9, 9, 6], [6, 9, 9, 6], [4, 6, 6, 4]]) * 2.0
+    assert np.array_equal(got, inside)
