@@ -253,6 +253,36 @@ CRISP_API crisp_status_t crisp_decode(crisp_handle_t h, uint16_t *d_w_dense_bf16
 CRISP_API crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ldx,
                                     int64_t ncols, void *d_y, int64_t ldy, int32_t y_dtype, void *stream);
 
+/*
+ * The same product for a convolution layer without materialising X (Sec. III, Notation: the
+ * K x K x R x S filter bank is the matrix W with one row per output channel; Sec. III-E step 1
+ * loads "the input activations corresponding to the non-zero blocks").  The reduction index of W
+ * is ordered (kernel row, kernel column, input channel), channel fastest, so a kept k-block of
+ * block_k channels lies inside one filter tap, and its activations are a shifted window of the
+ * input: they are fetched on the fly from the NHWC activation, the zero padding included.
+ *
+ *   Y[s, b, y, x] = sum_(i, j, r) W_hybrid[s, (i*kernel_w + j)*channels + r]
+ *                                 * A[b, y + i - pad, x + j - pad, r]        (stride 1)
+ *
+ *   d_act_nhwc  [batch, height, width, channels] bf16, dense, 16-byte aligned
+ *   d_y         [rows, batch*ho*wo] bf16 (y_dtype 0) or fp32 (1), leading dimension ldy,
+ *               ho = height + 2*pad - kernel_h + 1, wo likewise
+ * The handle's k must equal kernel_h*kernel_w*channels (BAD_SHAPE otherwise).  Supported
+ * (UNSUPPORTED otherwise; lower the convolution to a matrix and call crisp_spmm): block_k = 64,
+ * channels a multiple of 64, wo*sizeof(Y element) and ldy*sizeof(Y element) multiples of 16
+ * bytes, a tensor-core execution image and at least one kept block.  Same tolerance and status
+ * reporting as crisp_spmm.
+ */
+typedef struct {
+    int32_t batch, height, width, channels;   /* input activation, NHWC                         */
+    int32_t kernel_h, kernel_w;               /* filter taps                                    */
+    int32_t pad;                              /* zero padding on every side                     */
+} crisp_conv_desc_t;
+
+CRISP_API crisp_status_t crisp_spmm_conv(crisp_handle_t handle, const uint16_t *d_act_nhwc,
+                                         const crisp_conv_desc_t *conv, void *d_y, int64_t ldy,
+                                         int32_t y_dtype, void *stream);
+
 /* Restrict crisp_spmm of this handle to one kernel family (CRISP_PATH_*), or -1 for the
  * default choice.  UNSUPPORTED if the handle's execution image cannot serve that path. */
 CRISP_API crisp_status_t crisp_set_path(crisp_handle_t h, int32_t path);

@@ -29,6 +29,11 @@ class RankLayer(C.Structure):
                 ("block_elems", C.c_int64), ("min_keep", C.c_int32), ("reserved", C.c_int32)]
 
 
+class ConvDesc(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("height", C.c_int32), ("width", C.c_int32), ("channels", C.c_int32),
+                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad", C.c_int32)]
+
+
 class BytesModel(C.Structure):
     _fields_ = [("nnz", C.c_int64), ("vals_bytes", C.c_int64), ("idx_bytes", C.c_int64),
                 ("blk_col_bytes", C.c_int64), ("x_bytes", C.c_int64), ("y_bytes", C.c_int64),
@@ -74,6 +79,7 @@ def load(path: Optional[str] = None):
         "crisp_export": [vp, vp, vp, vp, vp],
         "crisp_decode": [vp, vp, i64, vp],
         "crisp_spmm": [vp, vp, i64, i64, vp, i64, i32, vp],
+        "crisp_spmm_conv": [vp, vp, P(ConvDesc), vp, i64, i32, vp],
         "crisp_set_path": [vp, i32],
         "crisp_device_status": [vp, vp, P(i32)],
         "crisp_bytes_model": [vp, i64, i32, P(BytesModel)],
@@ -235,6 +241,11 @@ def crisp_spmm(handle: int, d_x, ldx: int, ncols: int, d_y, ldy: int, y_dtype: i
     _check(load().crisp_spmm(handle, _ptr(d_x), ldx, ncols, _ptr(d_y), ldy, y_dtype, _stream(stream)), "crisp_spmm")
 
 
+def crisp_spmm_conv(handle: int, d_act_nhwc, conv: ConvDesc, d_y, ldy: int, y_dtype: int = 0, stream=None):
+    _check(load().crisp_spmm_conv(handle, _ptr(d_act_nhwc), C.byref(conv), _ptr(d_y), ldy, y_dtype, _stream(stream)),
+           "crisp_spmm_conv")
+
+
 def crisp_set_path(handle: int, path: int):
     _check(load().crisp_set_path(handle, path), "crisp_set_path")
 
@@ -349,6 +360,19 @@ class HybridLayer:
             y = torch.empty((self.desc.rows, ncols), dtype=torch.float32 if y_dtype else torch.bfloat16,
                             device=self.device)
         crisp_spmm(self.handle, x, x.stride(0), ncols, y, y.stride(0), y_dtype, stream)
+        return y
+
+    def spmm_conv(self, act_nhwc, kernel_h, kernel_w, pad, y=None, y_dtype=0, stream=None):
+        """Convolution (stride 1) of an NHWC bf16 activation with this layer's weights, without an X matrix."""
+        torch = self.torch
+        assert act_nhwc.is_cuda and act_nhwc.element_size() == 2 and act_nhwc.is_contiguous() and act_nhwc.dim() == 4
+        b, h, w, c = act_nhwc.shape
+        ho, wo = h + 2 * pad - kernel_h + 1, w + 2 * pad - kernel_w + 1
+        if y is None:
+            y = torch.empty((self.desc.rows, b * ho * wo), dtype=torch.float32 if y_dtype else torch.bfloat16,
+                            device=self.device)
+        crisp_spmm_conv(self.handle, act_nhwc, ConvDesc(b, h, w, c, kernel_h, kernel_w, pad), y, y.stride(0),
+                        y_dtype, stream)
         return y
 
     def set_path(self, path: int):

@@ -253,8 +253,35 @@ crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ld
                                            ncols, d_y, ldy, y_dtype, (cudaStream_t)stream);
         else
         e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx, ncols,
-                                  d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, (cudaStream_t)stream);
+                                  d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, nullptr, (cudaStream_t)stream);
     }
+    return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
+}
+
+crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, const crisp_conv_desc_t *cd, void *d_y,
+                               int64_t ldy, int32_t y_dtype, void *stream) {
+    if (!h || !d_act_nhwc || !cd || !d_y) return CRISP_INVALID_ARG;
+    if (y_dtype != 0 && y_dtype != 1) return CRISP_INVALID_ARG;
+    if (cd->batch <= 0 || cd->height <= 0 || cd->width <= 0 || cd->channels <= 0 || cd->kernel_h <= 0 ||
+        cd->kernel_w <= 0 || cd->pad < 0)
+        return CRISP_BAD_SHAPE;
+    crisp::ConvGeom cg{cd->batch, cd->height, cd->width, cd->channels, cd->kernel_h, cd->kernel_w, cd->pad,
+                       cd->height + 2 * cd->pad - cd->kernel_h + 1, cd->width + 2 * cd->pad - cd->kernel_w + 1};
+    if (cg.ho <= 0 || cg.wo <= 0) return CRISP_BAD_SHAPE;
+    if ((int64_t)cd->kernel_h * cd->kernel_w * cd->channels != h->g.k) return CRISP_BAD_SHAPE;
+    const int64_t ncols = (int64_t)cg.batch * cg.ho * cg.wo;
+    if (ldy < ncols) return CRISP_BAD_SHAPE;
+    const int es = y_dtype ? 4 : 2;
+    // the gather needs whole k-blocks inside one filter tap, 128-byte channel slabs, and TMA-addressable tensors
+    if (h->g.bk != 64 || cd->channels % h->g.bk != 0) return CRISP_UNSUPPORTED;
+    if (((int64_t)cg.wo * es) % 16 != 0 || (ldy * es) % 16 != 0 || !aligned(d_act_nhwc, 16) || !aligned(d_y, 16))
+        return CRISP_UNSUPPORTED;
+    const int path = h->forced_path >= 0 ? h->forced_path : h->exec_kind;
+    if (path == CRISP_PATH_DIRECT || h->g.kkeep == 0) return CRISP_UNSUPPORTED;
+    const char *nt = std::getenv("CRISP_TC_NT");
+    cudaError_t e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_act_nhwc, 0, ncols,
+                                          d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, &cg, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return CRISP_UNSUPPORTED;
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }
 

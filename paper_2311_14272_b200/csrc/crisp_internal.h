@@ -84,9 +84,12 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
 cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, cudaStream_t st);
 bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols);
+// Convolution geometry for the implicit-GEMM mode (stride 1): NHWC activation, ho x wo output pixels.
+struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo; };
+// conv == nullptr: d_x is the [k, ncols] matrix.  Otherwise d_x is the activation and ncols = batch*ho*wo.
 cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
                            const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
-                           int nt_override, cudaStream_t st);
+                           int nt_override, const ConvGeom *conv, cudaStream_t st);
 // spmm_tc_pair.cu: two CTAs (cta_group::2) share the X tile of the union of two adjacent CTA tiles' lists
 bool tc_pair_supported(const Geometry &g, int64_t ncols);
 cudaError_t launch_spmm_tc_pair(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,

@@ -36,7 +36,18 @@ struct TcParams {
     uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
     uint32_t stg_bufs;          // staging tiles per epilogue warp (1, 2 or 4): stores in flight per warp
     uint32_t stg_tile_bytes;    // one staging tile: 16 or 32 rows of 128 bytes (= the row count of map_y's box)
+    uint32_t stg_swz_mask;      // 16-byte chunk j of staging row r sits at j ^ (r & mask): 7 = 128-byte swizzle of
+                                // map_y, 3 / 1 / 0 = 64-byte / 32-byte / none (convolution: span = inner box bytes)
     uint32_t walk_cache;        // walk lists are copied into shared memory at kernel start
+    // Convolution as implicit GEMM: X is not a matrix in memory but an NHWC activation; a column tile is a
+    // box of tw x th x tb output pixels and the X tile of a kept block (one filter tap, bk channels) is the
+    // same box of the activation shifted by the tap, fetched by one 4-D TMA load (zero fill = zero padding).
+    int conv;
+    int cv_tw, cv_th, cv_tb;    // pixel box of a column tile (tw * th * tb = tile columns)
+    int cv_tiles_x, cv_tiles_y; // column tiles per image row / per image column
+    int cv_cpt;                 // k-blocks per filter tap = channels / bk
+    int cv_kw, cv_pad;          // filter width, zero padding
+    int cv_wo, cv_ho, cv_batch; // output width, height, images
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
@@ -45,14 +56,39 @@ constexpr uint32_t kWideStageBytes = 2048;                      // epilogue stag
 // Epilogue warps: two per TMEM lane quarter, or four where short walks make the epilogue the longest role.
 // Threads: warp 0 producer, warp 1 MMA issuer, then the epilogue warps.
 
+// Where a tile's columns start: the first column (matrix mode) or the first output pixel (x, y, image) of
+// the tile's box (convolution mode).
+struct TileOrigin { int x, y, b; };
+
+__device__ __forceinline__ TileOrigin tile_origin(const TcParams &p, int ct, int tile_n) {
+    TileOrigin o;
+    if (!p.conv) { o.x = ct * tile_n; o.y = 0; o.b = 0; return o; }
+    const int per_image = p.cv_tiles_x * p.cv_tiles_y;
+    const int bb = ct / per_image, r = ct - bb * per_image;
+    const int by = r / p.cv_tiles_x;
+    o.x = (r - by * p.cv_tiles_x) * p.cv_tw; o.y = by * p.cv_th; o.b = bb * p.cv_tb;
+    return o;
+}
+
 // One epilogue chunk: 32 rows (one per lane) x 128 bytes.  Through the warp's 128B-swizzled staging
 // tile and a TMA store, or, where TMA cannot clip exactly (it clips at 16-byte granularity), with
 // guarded plain stores.
 template <typename OutT>
 __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap *map_y, uint32_t stg, uint8_t *stg_gen,
-                                            int lane, const uint32_t (&out)[32], int x0, int y0, uint32_t &slot) {
+                                            int lane, const uint32_t (&out)[32], const TileOrigin &org, int col0, int y0,
+                                            uint32_t &slot) {
     constexpr int kOutCols = 128 / (int)sizeof(OutT);
-    if (x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
+    const int x0 = org.x + col0;             // matrix mode: first column of the chunk
+    // convolution mode: the chunk is kOutCols / tw rows of tw pixels inside one image of the tile's box
+    int cx = 0, cy = 0, cb = 0;
+    bool inside = x0 < p.ncols;
+    if (p.conv) {
+        const int per_image = p.cv_tw * p.cv_th;
+        const int img = col0 / per_image;
+        cx = org.x; cy = org.y + (col0 - img * per_image) / p.cv_tw; cb = org.b + img;
+        inside = cx < p.cv_wo && cy < p.cv_ho && cb < p.cv_batch;
+    }
+    if (!p.conv && x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
         const int row = y0 + lane;
         if (row < p.rows && x0 < p.ncols) {
             OutT *dst = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy + x0;
@@ -84,14 +120,17 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         if (passes == 1 || (lane >> 4) == h) {
             uint8_t *tile = stg_gen + tile_off + (passes == 1 ? lane : (lane & 15)) * 128;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)          // 128B swizzle: 16-byte chunk j of row r sits at j ^ (r % 8)
-                *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
+            for (int j = 0; j < 8; ++j)          // map_y's swizzle: 16-byte chunk j of row r sits at j ^ (r & mask)
+                *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & p.stg_swz_mask)) << 4)) =
                     make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
         }
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-            if (x0 < p.ncols) tma_store_2d(map_y, stg + tile_off, x0, y0 + 16 * h);
+            if (inside) {
+                if (p.conv) tma_store_4d(map_y, stg + tile_off, cx, cy, cb, y0 + 16 * h);
+                else tma_store_2d(map_y, stg + tile_off, x0, y0 + 16 * h);
+            }
             bulk_commit();
         }
         slot = (slot + 1) & (p.stg_bufs - 1);
@@ -111,9 +150,14 @@ struct MmaRoleArgs {
 };
 template <int kTileN, bool kSparse, int kAccStages, int NM>
 __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a) {
-    constexpr uint32_t kIdesc = make_idesc(kTileN, kSparse);
+    // matrix mode: X rows are columns-contiguous (MN-major operand, 64-column boxes box_bytes apart, a K
+    // step is 32 or 16 rows); convolution mode: the activation tile is [pixel][bk channels] with the channels
+    // contiguous (K-major operand, 128-byte rows in 1024-byte groups of 8, a K step is 64 or 32 bytes)
+    const uint32_t idesc = p.conv ? (make_idesc(kTileN, kSparse) & ~(1u << 16)) : make_idesc(kTileN, kSparse);
     const uint64_t a_desc0 = make_smem_desc(a.ring, 2048, 128, kLayoutNone);
-    const uint64_t b_desc0 = make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
+    const uint64_t b_desc0 = p.conv ? make_smem_desc(a.ring + p.entry_bytes, 16, 1024, kLayoutSw128)
+                                    : make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
+    const uint32_t b_step = p.conv ? (kSparse ? 4u : 2u) : (kSparse ? 256u : 128u);
     const uint64_t m_desc0 = make_smem_desc(a.ring + p.a_bytes, 128, 128, kLayoutNone);
     const uint32_t stage_step = p.stage_bytes >> 4, ring_span = p.num_stages * stage_step;
     uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
@@ -133,12 +177,12 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
                 tmem_copy_128x128b(meta_tmem, m_desc0 + off);
 #pragma unroll
                 for (int j = 0; j < NM; ++j)
-                    mma_sparse(d_tmem, ad + j * 256, bd + j * 256, kIdesc | (uint32_t)(j & 1), accum | (uint32_t)j,
+                    mma_sparse(d_tmem, ad + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), accum | (uint32_t)j,
                                meta_tmem + (j & ~1));
                 meta_buf ^= 1u;
             } else {
 #pragma unroll
-                for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * 128, kIdesc, accum | (uint32_t)j);
+                for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * b_step, idesc, accum | (uint32_t)j);
             }
             accum = 1u;
             mma_commit(empty);                      // stage reusable once these MMAs have read it
@@ -231,6 +275,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int len = walk_len[st];
                 const int32_t *cols = walk_col + (int64_t)st * p.wcap;
                 const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
+                const TileOrigin org = tile_origin(p, ct, kTileN);
                 int arow = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
                 // The block column of entry e is a load in this thread's serial loop; left where it is used
                 // it costs a round trip per stage.  Keep the next kAhead in registers.
@@ -243,11 +288,20 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     for (int u = 0; u < kAhead; ++u) {
                         const int e = e0 + u;
                         if (e >= len) break;
-                        const int krow = col_q[u] * p.bk;
+                        const int jb = col_q[u];
+                        const int krow = jb * p.bk;
                         if (e + kAhead < len) col_q[u] = cols[e + kAhead];
                         if (!mbar_wait(empty, ph ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_expect_tx(full, tx_bytes);
-                        if (tiled) {
+                        if (p.conv) {
+                            // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box shifted
+                            // by the tap; pixels outside the image read as zero (the convolution's padding)
+                            const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
+                            const int ti = tap / p.cv_kw, tj = tap - ti * p.cv_kw;
+                            tma_load_2d(dst, &map_a, 0, arow, full);
+                            tma_load_4d(dst + p.entry_bytes, &map_x, c0, org.x + tj - p.cv_pad, org.y + ti - p.cv_pad, org.b, full);
+                            arow += (int)entry_rows;
+                        } else if (tiled) {
                             // tiled loads pipeline (untiled bulk copies are served one at a time): the weight
                             // tile comes in as a box of 256-byte image rows, the NT boxes of X as one 3-D load
                             tma_load_2d(dst, &map_a, 0, arow, full);
@@ -316,6 +370,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             tc_fence_after();
             const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
             const int y0 = st * kTileM + 32 * q;
+            const TileOrigin org = tile_origin(p, ct, kTileN);
             if (y0 >= p.rows) {
                 // this lane quarter lies below the last row of W: nothing to drain
                 tc_fence_before();
@@ -341,7 +396,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 32; ++i) out[i] = accr[c * 32 + i];
                     }
-                    store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + half * kWarpCols + c * kOutCols, y0, slot);
+                    store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, org, half * kWarpCols + c * kOutCols, y0, slot);
                 }
             } else {
                 if (half == 0) {
@@ -362,7 +417,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             tmem_ld32(t_addr + c * 32, out);
                             tmem_ld_wait();
                         }
-                        store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, ct * kTileN + c * kOutCols, y0, slot);
+                        store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0, slot);
                     }
                 }
                 tc_fence_before();
@@ -646,6 +701,25 @@ bool make_map_image(CUtensorMap *map, const void *image, uint64_t total_bytes, u
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A 4-D tiled map (dims/box innermost first, strides of dimensions 1..3 in bytes).  The swizzle span is the
+// inner box: 128, 64 or 32 bytes, none for 16.  (A store through a map whose span is wider than its inner
+// box raised an illegal memory access on B200, although the map encodes.)
+bool make_map_4d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, const uint64_t (&dims)[4],
+                 const uint64_t (&strides_bytes)[3], const uint32_t (&box)[4]) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    const uint64_t inner = (uint64_t)box[0] * elem_bytes;
+    if (!fn || (inner != 128 && inner != 64 && inner != 32 && inner != 16)) return false;
+    const CUtensorMapSwizzle swz = inner == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                 : inner == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    cuuint64_t d[4] = {dims[0], dims[1], dims[2], dims[3]};
+    cuuint64_t sb[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
+    cuuint32_t b[4] = {box[0], box[1], box[2], box[3]};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, dt, 4, const_cast<void *>(base), d, sb, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool tensor_maps_available() { return encode_tiled_fn() != nullptr; }
 
 }  // namespace tc
@@ -713,7 +787,7 @@ bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int 
 
 cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
                            const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
-                           int nt_override, cudaStream_t st) {
+                           int nt_override, const ConvGeom *conv, cudaStream_t st) {
     const TcImageLayout L = tc_image_layout(g, sparse);
     static int sm_count = 0;
     if (!sm_count) {
@@ -735,14 +809,40 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     // box and lane quarter; under the sparse image three boxes, so that two accumulators fit beside the
     // metadata columns and the next tile's MMAs do not wait for the drain.
     const bool short_walk = L.wcap <= 8 && nt_override <= 0;
-    if (short_walk && L.wcap <= 2 && sparse && nt == 4) nt = 3;
-    TcParams p;
+    if (short_walk && L.wcap <= 2 && sparse && nt == 4 && !conv) nt = 3;
+    TcParams p = {};
+    if (conv) {
+        // Pixel box of a column tile: tw * th * tb = 256 (or 128) output pixels, tw a power of two that divides
+        // a 128-byte staging row, whole staging rows per image.  Among the shapes that fit, the one that
+        // covers the fewest pixels outside the images wins (then the widest, then the tallest).
+        if (nt == 3) nt = 4;
+        if (nt < 2) nt = 2;
+        const int f32c = y_dtype != 0 ? 32 : 64;
+        int64_t best = -1;
+        for (int tw = 32; tw >= 8; tw >>= 1)
+            for (int th = 32; th >= 1; th >>= 1) {
+                const int n_tile = nt * kBoxN;
+                if (n_tile % (tw * th) != 0 || f32c % tw != 0 || (tw * th) % f32c != 0) continue;
+                const int tb = n_tile / (tw * th);
+                const int64_t covered = (int64_t)((conv->wo + tw - 1) / tw) * tw * ((conv->ho + th - 1) / th) * th *
+                                        ((conv->batch + tb - 1) / tb) * tb;
+                if (best < 0 || covered < best) { best = covered; p.cv_tw = tw; p.cv_th = th; p.cv_tb = tb; }
+            }
+        if (best < 0) return cudaErrorInvalidValue;
+        p.conv = 1;
+        p.cv_tiles_x = (conv->wo + p.cv_tw - 1) / p.cv_tw;
+        p.cv_tiles_y = (conv->ho + p.cv_th - 1) / p.cv_th;
+        p.cv_cpt = conv->channels / g.bk;
+        p.cv_kw = conv->kw; p.cv_pad = conv->pad;
+        p.cv_wo = conv->wo; p.cv_ho = conv->ho; p.cv_batch = conv->batch;
+    }
     p.image = d_exec + L.image_off;
     p.walk_col = reinterpret_cast<const int32_t *>(d_exec + L.walk_col_off);
     p.walk_len = reinterpret_cast<const int32_t *>(d_exec + L.walk_len_off);
     p.status = d_status;
     p.nst = L.nst; p.wcap = L.wcap; p.bk = g.bk; p.rows = g.rows; p.ncols = ncols; p.y = d_y; p.ldy = ldy;
     p.n_col_tiles = (int)((ncols + nt * kBoxN - 1) / (nt * kBoxN));
+    if (conv) p.n_col_tiles = p.cv_tiles_x * p.cv_tiles_y * ((conv->batch + p.cv_tb - 1) / p.cv_tb);
     const int64_t tiles = (int64_t)p.n_col_tiles * L.nst;
     if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
     p.num_tiles = (int)tiles;
@@ -775,15 +875,32 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     CUtensorMap mx, my, ma;
     p.a_map = make_map_image(&ma, p.image, (uint64_t)L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
     if (!p.a_map) ma = CUtensorMap{};
-    p.x_map_3d = (ncols % kBoxN == 0) &&
-                 make_map_x3d(&mx, d_x, (uint64_t)ncols, (uint64_t)g.k, (uint64_t)ldx, (uint32_t)g.bk, (uint32_t)nt);
-    if (!p.x_map_3d && !make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, (uint64_t)ncols, (uint64_t)g.k,
-                                    (uint64_t)ldx, kBoxN, (uint32_t)g.bk))
-        return cudaErrorInvalidValue;
     const bool f32 = y_dtype != 0;
-    if (!make_map_2d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, f32 ? 4 : 2, d_y,
-                     (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, p.stg_tile_bytes / 128))
-        return cudaErrorInvalidValue;
+    p.stg_swz_mask = 7;
+    if (conv) {
+        p.stg_swz_mask = (uint32_t)(p.cv_tw * (f32 ? 4 : 2)) / 16 - 1;      // 128 / 64 / 32 / 16-byte inner box of map_y
+        // activation [batch][height][width][channels] and Y [rows][batch][ho][wo] as 4-D tensors
+        if (!p.a_map) return cudaErrorInvalidValue;
+        p.x_map_3d = 0;
+        const uint64_t c = (uint64_t)conv->channels, w = (uint64_t)conv->width, h = (uint64_t)conv->height;
+        const uint64_t xd[4] = {c, w, h, (uint64_t)conv->batch}, xs[3] = {c * 2, w * c * 2, h * w * c * 2};
+        const uint32_t xb[4] = {(uint32_t)g.bk, (uint32_t)p.cv_tw, (uint32_t)p.cv_th, (uint32_t)p.cv_tb};
+        if (!make_map_4d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, xd, xs, xb)) return cudaErrorInvalidValue;
+        const uint64_t es = f32 ? 4 : 2, wo = (uint64_t)conv->wo, ho = (uint64_t)conv->ho;
+        const uint64_t yd[4] = {wo, ho, (uint64_t)conv->batch, (uint64_t)g.rows}, ys[3] = {wo * es, ho * wo * es, (uint64_t)ldy * es};
+        const uint32_t yb[4] = {(uint32_t)p.cv_tw, (uint32_t)((f32 ? 32 : 64) / p.cv_tw), 1u, p.stg_tile_bytes / 128};
+        if (!make_map_4d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (int)es, d_y, yd, ys, yb))
+            return cudaErrorInvalidValue;
+    } else {
+        p.x_map_3d = (ncols % kBoxN == 0) &&
+                     make_map_x3d(&mx, d_x, (uint64_t)ncols, (uint64_t)g.k, (uint64_t)ldx, (uint32_t)g.bk, (uint32_t)nt);
+        if (!p.x_map_3d && !make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, (uint64_t)ncols, (uint64_t)g.k,
+                                        (uint64_t)ldx, kBoxN, (uint32_t)g.bk))
+            return cudaErrorInvalidValue;
+        if (!make_map_2d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, f32 ? 4 : 2, d_y,
+                         (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, p.stg_tile_bytes / 128))
+            return cudaErrorInvalidValue;
+    }
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
 
 #define CRISP_TC_LAUNCH_E(NTV, SP, ACC, EPI)                                                              \
