@@ -280,6 +280,65 @@ def measure_global_rank(torch, B, dev, with_oracle, iters=12):
     return out
 
 
+_VGG_CONV = {1: (64, 224), 2: (64, 112), 3: (128, 112)}     # config-3 layer index -> (input channels, side)
+
+
+def measure_conv(torch, B, dev, peaks, flush_l2, iters=9):
+    """Convolution as implicit GEMM (crisp_spmm_conv on the NHWC activation) beside the same layer run as
+    crisp_spmm on the lowered K x Nc matrix and beside dense cuBLAS on that matrix: the three largest VGG-16
+    layers of config 3 (batch 16).  Roofline terms of the implicit call: the activation is read once."""
+    out = []
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        ts = []
+        for i in range(3 + iters):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        return float(np.mean(ts))
+
+    cfg = wl.config3()
+    for idx, (cin, side) in _VGG_CONV.items():
+        layer, batch = cfg[idx], 16
+        w = wl.make_weight(layer)
+        s = wl.make_saliency(layer, w)
+        d_w = torch.from_numpy(w.view(np.int16)).to(dev).view(torch.bfloat16)
+        g = torch.Generator(device=dev); g.manual_seed(layer.seed + 7)
+        act = torch.randn((batch, side, side, cin), device=dev, generator=g).clamp_(min=0).to(torch.bfloat16)
+        L = B.HybridLayer(layer.rows, layer.k, layer.n, layer.m, layer.block_rows, layer.block_k, layer.keep_ratio,
+                          device=dev)
+        L.build_mask(torch.from_numpy(s).to(dev)).encode(d_w)
+        ncols = batch * side * side
+        y = torch.empty((layer.rows, ncols), dtype=torch.bfloat16, device=dev)
+        y2 = torch.empty_like(y)
+        ms_i = timed(lambda: L.spmm_conv(act, 3, 3, 1, y=y))
+        ap = torch.nn.functional.pad(act, (0, 0, 1, 1, 1, 1))
+        x = torch.stack([ap[:, i:i + side, j:j + side, :] for i in range(3) for j in range(3)], dim=0) \
+            .permute(0, 4, 1, 2, 3).reshape(9 * cin, ncols).contiguous()
+        del ap
+        ms_e = timed(lambda: L.spmm(x, y=y2))
+        ms_d = timed(lambda: torch.matmul(d_w, x, out=y2))
+        L.spmm(x, y=y2)
+        torch.cuda.synchronize()
+        m = L.bytes_model(ncols)
+        alg = m["vals_bytes"] + m["idx_bytes"] + m["blk_col_bytes"] + act.numel() * 2 + m["y_bytes"]
+        t_hbm = alg / (peaks["hbm_gbs"] * 1e9)
+        r = roofline_terms(m, peaks, ms_i, ncols)
+        out.append({"workload": layer.name, "activation": [batch, side, side, cin], "kkeep": L.kkeep,
+                    "conv_us": ms_i * 1e3, "lowered_spmm_us": ms_e * 1e3, "dense_cublas_lowered_us": ms_d * 1e3,
+                    "speedup_vs_lowered": ms_e / ms_i, "speedup_vs_dense_cublas": ms_d / ms_i,
+                    "algorithmic_bytes": int(alg), "t_hbm_us": t_hbm * 1e6, "t_tensor_us": r["t_tensor"] * 1e6,
+                    "roofline_frac": max(t_hbm, r["t_tensor"]) / (ms_i * 1e-3),
+                    "identical_to_lowered": bool(torch.equal(y, y2)), "device_status": L.device_status()})
+        L.close()
+        del x, y, y2, act
+    return out
+
+
 def recorded_traffic(workload, kernel):
     """DRAM bytes per launch from the committed ncu capture, or None when the kernel source has
     changed since the counters were taken."""
@@ -467,6 +526,7 @@ def run_ours(args, layer, rank, world):
     if rank == 0 and world == 1 and not args.no_cells and args.workload.startswith("sweep_"):
         out["cells"] = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
         out["global_rank"] = measure_global_rank(torch, B, dev, not args.no_cpu_baseline)
+        out["conv"] = measure_conv(torch, B, dev, peaks, flush_l2)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)

@@ -60,9 +60,10 @@ constexpr uint32_t kWideStageBytes = 2048;                      // epilogue stag
 // the tile's box (convolution mode).
 struct TileOrigin { int x, y, b; };
 
+template <bool kConv>
 __device__ __forceinline__ TileOrigin tile_origin(const TcParams &p, int ct, int tile_n) {
     TileOrigin o;
-    if (!p.conv) { o.x = ct * tile_n; o.y = 0; o.b = 0; return o; }
+    if constexpr (!kConv) { o.x = ct * tile_n; o.y = 0; o.b = 0; return o; }
     const int per_image = p.cv_tiles_x * p.cv_tiles_y;
     const int bb = ct / per_image, r = ct - bb * per_image;
     const int by = r / p.cv_tiles_x;
@@ -73,7 +74,7 @@ __device__ __forceinline__ TileOrigin tile_origin(const TcParams &p, int ct, int
 // One epilogue chunk: 32 rows (one per lane) x 128 bytes.  Through the warp's 128B-swizzled staging
 // tile and a TMA store, or, where TMA cannot clip exactly (it clips at 16-byte granularity), with
 // guarded plain stores.
-template <typename OutT>
+template <typename OutT, bool kConv>
 __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap *map_y, uint32_t stg, uint8_t *stg_gen,
                                             int lane, const uint32_t (&out)[32], const TileOrigin &org, int col0, int y0,
                                             uint32_t &slot) {
@@ -82,13 +83,13 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
     // convolution mode: the chunk is kOutCols / tw rows of tw pixels inside one image of the tile's box
     int cx = 0, cy = 0, cb = 0;
     bool inside = x0 < p.ncols;
-    if (p.conv) {
+    if constexpr (kConv) {
         const int per_image = p.cv_tw * p.cv_th;
         const int img = col0 / per_image;
         cx = org.x; cy = org.y + (col0 - img * per_image) / p.cv_tw; cb = org.b + img;
         inside = cx < p.cv_wo && cy < p.cv_ho && cb < p.cv_batch;
     }
-    if (!p.conv && x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
+    if (!kConv && x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
         const int row = y0 + lane;
         if (row < p.rows && x0 < p.ncols) {
             OutT *dst = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy + x0;
@@ -121,14 +122,14 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
             uint8_t *tile = stg_gen + tile_off + (passes == 1 ? lane : (lane & 15)) * 128;
 #pragma unroll
             for (int j = 0; j < 8; ++j)          // map_y's swizzle: 16-byte chunk j of row r sits at j ^ (r & mask)
-                *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & p.stg_swz_mask)) << 4)) =
+                *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & (kConv ? p.stg_swz_mask : 7u))) << 4)) =
                     make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
         }
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
             if (inside) {
-                if (p.conv) tma_store_4d(map_y, stg + tile_off, cx, cy, cb, y0 + 16 * h);
+                if constexpr (kConv) tma_store_4d(map_y, stg + tile_off, cx, cy, cb, y0 + 16 * h);
                 else tma_store_2d(map_y, stg + tile_off, x0, y0 + 16 * h);
             }
             bulk_commit();
@@ -148,16 +149,16 @@ struct MmaRoleArgs {
     const int32_t *walk_len;
     volatile int *abort_flag;
 };
-template <int kTileN, bool kSparse, int kAccStages, int NM>
+template <int kTileN, bool kSparse, int kAccStages, int NM, bool kConv>
 __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a) {
     // matrix mode: X rows are columns-contiguous (MN-major operand, 64-column boxes box_bytes apart, a K
     // step is 32 or 16 rows); convolution mode: the activation tile is [pixel][bk channels] with the channels
     // contiguous (K-major operand, 128-byte rows in 1024-byte groups of 8, a K step is 64 or 32 bytes)
-    const uint32_t idesc = p.conv ? (make_idesc(kTileN, kSparse) & ~(1u << 16)) : make_idesc(kTileN, kSparse);
+    constexpr uint32_t idesc = kConv ? (make_idesc(kTileN, kSparse) & ~(1u << 16)) : make_idesc(kTileN, kSparse);
     const uint64_t a_desc0 = make_smem_desc(a.ring, 2048, 128, kLayoutNone);
-    const uint64_t b_desc0 = p.conv ? make_smem_desc(a.ring + p.entry_bytes, 16, 1024, kLayoutSw128)
-                                    : make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
-    const uint32_t b_step = p.conv ? (kSparse ? 4u : 2u) : (kSparse ? 256u : 128u);
+    const uint64_t b_desc0 = kConv ? make_smem_desc(a.ring + p.entry_bytes, 16, 1024, kLayoutSw128)
+                                   : make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
+    constexpr uint32_t b_step = kConv ? (kSparse ? 4u : 2u) : (kSparse ? 256u : 128u);
     const uint64_t m_desc0 = make_smem_desc(a.ring + p.a_bytes, 128, 128, kLayoutNone);
     const uint32_t stage_step = p.stage_bytes >> 4, ring_span = p.num_stages * stage_step;
     uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
@@ -204,7 +205,7 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
 // contiguous, 128 bytes between 8-row groups, 2048 bytes between 16-byte K chunks.
 // X box layout: TMA SWIZZLE_128B, 64 columns (128 bytes) x bk rows; MN-major operand with 1024 bytes
 // between 8-row K groups and box_bytes between 64-column groups.
-template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi>
+template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi, bool kConv>
 __global__ void __launch_bounds__(64 + 32 * kEpi, 1)
 spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                const __grid_constant__ CUtensorMap map_a, TcParams p) {
@@ -275,7 +276,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int len = walk_len[st];
                 const int32_t *cols = walk_col + (int64_t)st * p.wcap;
                 const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
-                const TileOrigin org = tile_origin(p, ct, kTileN);
+                const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
                 int arow = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
                 // The block column of entry e is a load in this thread's serial loop; left where it is used
                 // it costs a round trip per stage.  Keep the next kAhead in registers.
@@ -293,7 +294,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         if (e + kAhead < len) col_q[u] = cols[e + kAhead];
                         if (!mbar_wait(empty, ph ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_expect_tx(full, tx_bytes);
-                        if (p.conv) {
+                        if constexpr (kConv) {
                             // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box shifted
                             // by the tap; pixels outside the image read as zero (the convolution's padding)
                             const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
@@ -334,17 +335,17 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             const int nmma = kSparse ? p.bk / 32 : p.bk / 16;        // K = 32 (sparse) or K = 16 steps per block
             if constexpr (kSparse) {
                 switch (nmma) {
-                    case 1: mma_role<kTileN, true, kAccStages, 1>(p, a); break;
-                    case 2: mma_role<kTileN, true, kAccStages, 2>(p, a); break;
-                    case 3: mma_role<kTileN, true, kAccStages, 3>(p, a); break;
-                    default: mma_role<kTileN, true, kAccStages, 4>(p, a); break;
+                    case 1: mma_role<kTileN, true, kAccStages, 1, kConv>(p, a); break;
+                    case 2: mma_role<kTileN, true, kAccStages, 2, kConv>(p, a); break;
+                    case 3: mma_role<kTileN, true, kAccStages, 3, kConv>(p, a); break;
+                    default: mma_role<kTileN, true, kAccStages, 4, kConv>(p, a); break;
                 }
             } else {
                 switch (nmma) {
-                    case 2: mma_role<kTileN, false, kAccStages, 2>(p, a); break;
-                    case 4: mma_role<kTileN, false, kAccStages, 4>(p, a); break;
-                    case 6: mma_role<kTileN, false, kAccStages, 6>(p, a); break;
-                    default: mma_role<kTileN, false, kAccStages, 8>(p, a); break;
+                    case 2: mma_role<kTileN, false, kAccStages, 2, kConv>(p, a); break;
+                    case 4: mma_role<kTileN, false, kAccStages, 4, kConv>(p, a); break;
+                    case 6: mma_role<kTileN, false, kAccStages, 6, kConv>(p, a); break;
+                    default: mma_role<kTileN, false, kAccStages, 8, kConv>(p, a); break;
                 }
             }
         }
@@ -370,7 +371,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             tc_fence_after();
             const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
             const int y0 = st * kTileM + 32 * q;
-            const TileOrigin org = tile_origin(p, ct, kTileN);
+            const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
             if (y0 >= p.rows) {
                 // this lane quarter lies below the last row of W: nothing to drain
                 tc_fence_before();
@@ -396,7 +397,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 32; ++i) out[i] = accr[c * 32 + i];
                     }
-                    store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, org, half * kWarpCols + c * kOutCols, y0, slot);
+                    store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, half * kWarpCols + c * kOutCols, y0, slot);
                 }
             } else {
                 if (half == 0) {
@@ -417,7 +418,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             tmem_ld32(t_addr + c * 32, out);
                             tmem_ld_wait();
                         }
-                        store_chunk<OutT>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0, slot);
+                        store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0, slot);
                     }
                 }
                 tc_fence_before();
@@ -625,10 +626,10 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
     for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = s_tile4[i];
 }
 
-template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi>
+template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi, bool kConv>
 cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const CUtensorMap &ma, const TcParams &p,
                            int grid, size_t smem, cudaStream_t st) {
-    auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi>;
+    auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi, kConv>;
     static size_t configured = 0;                       // largest dynamic shared memory opted into so far
     if (smem > configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -903,10 +904,19 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     }
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
 
-#define CRISP_TC_LAUNCH_E(NTV, SP, ACC, EPI)                                                              \
-    (f32 ? launch_variant<NTV, SP, ACC, float, EPI>(mx, my, ma, p, grid, smem, st)                            \
-         : launch_variant<NTV, SP, ACC, uint16_t, EPI>(mx, my, ma, p, grid, smem, st))
+#define CRISP_TC_LAUNCH_C(NTV, SP, ACC, EPI, CONV)                                                        \
+    (f32 ? launch_variant<NTV, SP, ACC, float, EPI, CONV>(mx, my, ma, p, grid, smem, st)                      \
+         : launch_variant<NTV, SP, ACC, uint16_t, EPI, CONV>(mx, my, ma, p, grid, smem, st))
+#define CRISP_TC_LAUNCH_E(NTV, SP, ACC, EPI) CRISP_TC_LAUNCH_C(NTV, SP, ACC, EPI, false)
 #define CRISP_TC_LAUNCH(NTV, SP, ACC) CRISP_TC_LAUNCH_E(NTV, SP, ACC, 8)
+    if (conv) {                              // the gather uses 128- or 256-pixel tiles only
+        if (sparse) {
+            if (nt == 2) return CRISP_TC_LAUNCH_C(2, true, 2, 8, true);
+            return epi == 16 ? CRISP_TC_LAUNCH_C(4, true, 1, 16, true) : CRISP_TC_LAUNCH_C(4, true, 1, 8, true);
+        }
+        if (nt == 2) return CRISP_TC_LAUNCH_C(2, false, 2, 8, true);
+        return epi == 16 ? CRISP_TC_LAUNCH_C(4, false, 2, 16, true) : CRISP_TC_LAUNCH_C(4, false, 2, 8, true);
+    }
     if (sparse) {
         switch (nt) {
             case 1: return CRISP_TC_LAUNCH(1, true, 2);
@@ -923,6 +933,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     }
 #undef CRISP_TC_LAUNCH
 #undef CRISP_TC_LAUNCH_E
+#undef CRISP_TC_LAUNCH_C
 }
 
 }  // namespace crisp
