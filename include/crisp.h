@@ -283,6 +283,18 @@ CRISP_API crisp_status_t crisp_spmm_conv(crisp_handle_t handle, const uint16_t *
                                          const crisp_conv_desc_t *conv, void *d_y, int64_t ldy,
                                          int32_t y_dtype, void *stream);
 
+/*
+ * Layer epilogue for every later crisp_spmm / crisp_spmm_conv on this handle:
+ *   Y = act(W_hybrid * X + bias),  act = max(., 0) when relu = 1, identity when 0,
+ * applied to the fp32 accumulator before the store, so a bf16 Y is rounded once and can be the
+ * next layer's X as it stands (pointwise layers: Y [rows, ncols] is the next X [k, ncols]).  The
+ * paper prunes whole networks (Sec. IV: ResNet-50, VGG-16, MobileNetV2), whose layers end in a
+ * bias (folded batch norm) and a ReLU; it gives no formula of its own for this step.
+ *   d_bias_f32  device, [rows] fp32, read at every call (the caller keeps it alive), or NULL
+ * (NULL, 0) restores the plain product.
+ */
+CRISP_API crisp_status_t crisp_set_epilogue(crisp_handle_t handle, const float *d_bias_f32, int32_t relu);
+
 /* Restrict crisp_spmm of this handle to one kernel family (CRISP_PATH_*), or -1 for the
  * default choice.  UNSUPPORTED if the handle's execution image cannot serve that path. */
 CRISP_API crisp_status_t crisp_set_path(crisp_handle_t h, int32_t path);

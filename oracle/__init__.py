@@ -223,3 +223,14 @@ def conv_fp64(w_dense: np.ndarray, kh: int, kw: int, act_bits: np.ndarray, pad: 
     if rc:
         raise ValueError(f"oracle_conv_fp64 rc={rc}")
     return y
+
+
+def bias_relu(y: np.ndarray, bias=None, relu: bool = False) -> np.ndarray:
+    """Layer epilogue on an fp64 product [rows, ncols]: + bias[row] (fp32 values), then max(., 0) if relu."""
+    out = np.ascontiguousarray(y, dtype=np.float64).copy()
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    rc = lib().oracle_bias_relu(_p(out, C.c_double), C.c_int(out.shape[0]), C.c_int64(out.shape[1]),
+                                _p(b, C.c_float), C.c_int(1 if relu else 0))
+    if rc:
+        raise ValueError(f"oracle_bias_relu rc={rc}")
+    return out

@@ -520,3 +520,22 @@ int oracle_conv_fp64(const double *w_dense, int s_out, int kh, int kw, int r_in,
                 }
     return 0;
 }
+
+/* -------------------------------------------------------------- layer epilogue */
+
+/*
+ * The step that closes a layer of the networks the paper prunes (Sec. IV): per output channel a
+ * bias, then optionally the rectifier.  In place on the fp64 product y [rows, ncols]:
+ *   y[r, c] = max(y[r, c] + bias[r], 0)   (the max only when relu != 0; bias may be NULL)
+ */
+int oracle_bias_relu(double *y, int rows, int64_t ncols, const float *bias, int relu)
+{
+    if (!y || rows <= 0 || ncols <= 0) return -1;
+    for (int r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < ncols; ++c) {
+            double v = y[(int64_t)r * ncols + c] + (bias ? (double)bias[r] : 0.0);
+            if (relu && v < 0.0) v = 0.0;
+            y[(int64_t)r * ncols + c] = v;
+        }
+    return 0;
+}

@@ -81,6 +81,7 @@ def load(path: Optional[str] = None):
         "crisp_spmm": [vp, vp, i64, i64, vp, i64, i32, vp],
         "crisp_spmm_conv": [vp, vp, P(ConvDesc), vp, i64, i32, vp],
         "crisp_set_path": [vp, i32],
+        "crisp_set_epilogue": [vp, vp, i32],
         "crisp_device_status": [vp, vp, P(i32)],
         "crisp_bytes_model": [vp, i64, i32, P(BytesModel)],
         "crisp_mask_scores": [P(LayerDesc), vp, P(vp), P(vp)],
@@ -246,6 +247,10 @@ def crisp_spmm_conv(handle: int, d_act_nhwc, conv: ConvDesc, d_y, ldy: int, y_dt
            "crisp_spmm_conv")
 
 
+def crisp_set_epilogue(handle: int, d_bias_f32, relu: int):
+    _check(load().crisp_set_epilogue(handle, _ptr(d_bias_f32), int(relu)), "crisp_set_epilogue")
+
+
 def crisp_set_path(handle: int, path: int):
     _check(load().crisp_set_path(handle, path), "crisp_set_path")
 
@@ -374,6 +379,14 @@ class HybridLayer:
         crisp_spmm_conv(self.handle, act_nhwc, ConvDesc(b, h, w, c, kernel_h, kernel_w, pad), y, y.stride(0),
                         y_dtype, stream)
         return y
+
+    def set_epilogue(self, bias=None, relu=False):
+        """Y = act(W X + bias) for later products; `bias` is an fp32 CUDA tensor [rows] that this object keeps."""
+        if bias is not None:
+            assert bias.is_cuda and bias.dtype == self.torch.float32 and bias.numel() == self.desc.rows
+        self._bias = bias
+        crisp_set_epilogue(self.handle, bias, 1 if relu else 0)
+        return self
 
     def set_path(self, path: int):
         crisp_set_path(self.handle, path)

@@ -174,6 +174,7 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     h->exec_kind = image_kind(g);
     h->exec_payload_bytes = exec_payload_bytes(g, h->exec_kind);
     h->forced_path = -1;
+    h->epilogue = crisp::Epilogue{nullptr, 0};
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
     // 128-row blocks: one kept block is one tensor-core tile, so the encode kernel writes it directly
@@ -222,6 +223,13 @@ crisp_status_t crisp_decode(crisp_handle_t h, uint16_t *d_w_dense_bf16, int64_t 
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }
 
+crisp_status_t crisp_set_epilogue(crisp_handle_t h, const float *d_bias_f32, int32_t relu) {
+    if (!h || (relu != 0 && relu != 1)) return CRISP_INVALID_ARG;
+    if (d_bias_f32 && !aligned(d_bias_f32, 4)) return CRISP_INVALID_ARG;
+    h->epilogue = crisp::Epilogue{d_bias_f32, relu};
+    return CRISP_OK;
+}
+
 crisp_status_t crisp_set_path(crisp_handle_t h, int32_t path) {
     if (!h) return CRISP_INVALID_ARG;
     if (path == -1 || path == CRISP_PATH_DIRECT) { h->forced_path = path; return CRISP_OK; }
@@ -243,17 +251,18 @@ crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ld
     cudaError_t e;
     if (path == CRISP_PATH_DIRECT) {
         e = crisp::launch_spmm_direct(h->g, h->d_blk_col, h->d_vals, h->d_idx, d_x_bf16, ldx, ncols,
-                                      d_y, ldy, y_dtype, (cudaStream_t)stream);
+                                      d_y, ldy, y_dtype, h->epilogue, (cudaStream_t)stream);
     } else {
         const char *pair = std::getenv("CRISP_TC_PAIR");   // 1: CTA-pair kernel, 0: single-CTA kernel
-        const bool use_pair = pair && std::atoi(pair) == 1 && crisp::tc_pair_supported(h->g, ncols);
+        const bool plain = h->epilogue.bias == nullptr && !h->epilogue.relu;      // the pair kernel has no layer epilogue
+        const bool use_pair = pair && std::atoi(pair) == 1 && plain && crisp::tc_pair_supported(h->g, ncols);
         const char *nt = std::getenv("CRISP_TC_NT");     // column boxes per CTA tile, tuning only
         if (use_pair)
             e = crisp::launch_spmm_tc_pair(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx,
                                            ncols, d_y, ldy, y_dtype, (cudaStream_t)stream);
         else
         e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx, ncols,
-                                  d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, nullptr, (cudaStream_t)stream);
+                                  d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, nullptr, h->epilogue, (cudaStream_t)stream);
     }
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }
@@ -280,7 +289,7 @@ crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, con
     if (path == CRISP_PATH_DIRECT || h->g.kkeep == 0) return CRISP_UNSUPPORTED;
     const char *nt = std::getenv("CRISP_TC_NT");
     cudaError_t e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_act_nhwc, 0, ncols,
-                                          d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, &cg, (cudaStream_t)stream);
+                                          d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, &cg, h->epilogue, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return CRISP_UNSUPPORTED;
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }

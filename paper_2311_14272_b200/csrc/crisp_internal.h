@@ -8,6 +8,12 @@
 
 namespace crisp {
 
+// Layer epilogue applied to the fp32 accumulator before the store: Y = act(W*X + bias).
+struct Epilogue {
+    const float *bias;      // device, [rows] fp32, or nullptr
+    int relu;               // max(., 0) after the bias
+};
+
 // Shape of one layer after padding to whole blocks.
 struct Geometry {
     int rows, k, n, m, bm, bk;
@@ -48,6 +54,7 @@ struct crisp_handle_s {
     size_t exec_payload_bytes;
     int exec_kind;          // CRISP_PATH_* the image was laid out for (DIRECT = none)
     int forced_path;        // -1 = default
+    crisp::Epilogue epilogue;
 };
 
 namespace crisp {
@@ -89,7 +96,7 @@ struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo; };
 // conv == nullptr: d_x is the [k, ncols] matrix.  Otherwise d_x is the activation and ncols = batch*ho*wo.
 cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
                            const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
-                           int nt_override, const ConvGeom *conv, cudaStream_t st);
+                           int nt_override, const ConvGeom *conv, const Epilogue &epi, cudaStream_t st);
 // spmm_tc_pair.cu: two CTAs (cta_group::2) share the X tile of the union of two adjacent CTA tiles' lists
 bool tc_pair_supported(const Geometry &g, int64_t ncols);
 cudaError_t launch_spmm_tc_pair(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
@@ -99,6 +106,6 @@ cudaError_t launch_spmm_tc_pair(const Geometry &g, bool sparse, const uint8_t *d
 // spmm_direct.cu
 cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, const uint16_t *d_x, int64_t ldx, int64_t ncols,
-                               void *d_y, int64_t ldy, int y_dtype, cudaStream_t st);
+                               void *d_y, int64_t ldy, int y_dtype, const Epilogue &epi, cudaStream_t st);
 
 }  // namespace crisp

@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(kTileN * kRowLanes)
 spmm_direct_kernel(Geometry g, const int32_t *__restrict__ blk_col,
                    const uint16_t *__restrict__ vals, const uint32_t *__restrict__ idx,
                    const uint16_t *__restrict__ x, int64_t ldx, int64_t ncols,
-                   OutT *__restrict__ y, int64_t ldy) {
+                   OutT *__restrict__ y, int64_t ldy, Epilogue epi) {
     extern __shared__ float xs[];                    // [bk][kTileN]
     const int tx = threadIdx.x % kTileN, ty = threadIdx.x / kTileN;
     const int rt = blockIdx.y;
@@ -69,10 +69,13 @@ spmm_direct_kernel(Geometry g, const int32_t *__restrict__ blk_col,
         for (int i = 0; i < kAcc; ++i) {
             const int64_t row = (int64_t)rt * BM + ty + i * kRowLanes;
             if (row < g.rows) {
+                float v = acc[i];
+                if (epi.bias) v += epi.bias[row];
+                if (epi.relu) v = fmaxf(v, 0.f);
                 if constexpr (sizeof(OutT) == 2)
-                    y[row * ldy + c0 + tx] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[i]));
+                    y[row * ldy + c0 + tx] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
                 else
-                    y[row * ldy + c0 + tx] = acc[i];
+                    y[row * ldy + c0 + tx] = v;
             }
         }
     }
@@ -81,15 +84,15 @@ spmm_direct_kernel(Geometry g, const int32_t *__restrict__ blk_col,
 template <typename OutT>
 cudaError_t launch_typed(const Geometry &g, const int32_t *bc, const uint16_t *vals, const uint32_t *idx,
                          const uint16_t *x, int64_t ldx, int64_t ncols, OutT *y, int64_t ldy,
-                         cudaStream_t st) {
+                         const Epilogue &epi, cudaStream_t st) {
     const int64_t gx = (ncols + kTileN - 1) / kTileN;
     const size_t smem = (size_t)g.bk * kTileN * sizeof(float);
     dim3 grid((unsigned)gx, (unsigned)g.nrt);
     const int threads = kTileN * kRowLanes;
     switch (g.bm) {
-        case 32: spmm_direct_kernel<32, OutT><<<grid, threads, smem, st>>>(g, bc, vals, idx, x, ldx, ncols, y, ldy); break;
-        case 64: spmm_direct_kernel<64, OutT><<<grid, threads, smem, st>>>(g, bc, vals, idx, x, ldx, ncols, y, ldy); break;
-        case 128: spmm_direct_kernel<128, OutT><<<grid, threads, smem, st>>>(g, bc, vals, idx, x, ldx, ncols, y, ldy); break;
+        case 32: spmm_direct_kernel<32, OutT><<<grid, threads, smem, st>>>(g, bc, vals, idx, x, ldx, ncols, y, ldy, epi); break;
+        case 64: spmm_direct_kernel<64, OutT><<<grid, threads, smem, st>>>(g, bc, vals, idx, x, ldx, ncols, y, ldy, epi); break;
+        case 128: spmm_direct_kernel<128, OutT><<<grid, threads, smem, st>>>(g, bc, vals, idx, x, ldx, ncols, y, ldy, epi); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
@@ -99,12 +102,12 @@ cudaError_t launch_typed(const Geometry &g, const int32_t *bc, const uint16_t *v
 
 cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, const uint16_t *d_x, int64_t ldx, int64_t ncols,
-                               void *d_y, int64_t ldy, int y_dtype, cudaStream_t st) {
+                               void *d_y, int64_t ldy, int y_dtype, const Epilogue &epi, cudaStream_t st) {
     if (y_dtype == 0)
         return launch_typed<uint16_t>(g, d_blk_col, d_vals, d_idx, d_x, ldx, ncols,
-                                      reinterpret_cast<uint16_t *>(d_y), ldy, st);
+                                      reinterpret_cast<uint16_t *>(d_y), ldy, epi, st);
     return launch_typed<float>(g, d_blk_col, d_vals, d_idx, d_x, ldx, ncols,
-                               reinterpret_cast<float *>(d_y), ldy, st);
+                               reinterpret_cast<float *>(d_y), ldy, epi, st);
 }
 
 }  // namespace crisp

@@ -48,6 +48,8 @@ struct TcParams {
     int cv_cpt;                 // k-blocks per filter tap = channels / bk
     int cv_kw, cv_pad;          // filter width, zero padding
     int cv_wo, cv_ho, cv_batch; // output width, height, images
+    const float *bias;          // layer epilogue: Y = act(W*X + bias); nullptr = no bias
+    int relu;
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
@@ -372,6 +374,10 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
             const int y0 = st * kTileM + 32 * q;
             const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
+            // layer epilogue on the fp32 accumulator: this lane's row gets its bias, then the activation
+            const bool fuse = p.bias != nullptr || p.relu != 0;
+            const float bias_v = (p.bias != nullptr && y0 + lane < p.rows) ? p.bias[y0 + lane] : 0.f;
+            const float floor_v = p.relu ? 0.f : -__int_as_float(0x7f800000);
             if (y0 >= p.rows) {
                 // this lane quarter lies below the last row of W: nothing to drain
                 tc_fence_before();
@@ -386,6 +392,11 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);       // accumulator free for the next tile
+                if (fuse) {
+#pragma unroll
+                    for (int i = 0; i < kWarpCols; ++i)
+                        accr[i] = __float_as_uint(fmaxf(__uint_as_float(accr[i]) + bias_v, floor_v));
+                }
 #pragma unroll
                 for (int c = 0; c < kWarpCols / kOutCols; ++c) {
                     uint32_t out[32];
@@ -409,6 +420,13 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             tmem_ld32(t_addr + c * 64, r0);
                             tmem_ld32(t_addr + c * 64 + 32, r1);
                             tmem_ld_wait();
+                            if (fuse) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) {
+                                    r0[i] = __float_as_uint(fmaxf(__uint_as_float(r0[i]) + bias_v, floor_v));
+                                    r1[i] = __float_as_uint(fmaxf(__uint_as_float(r1[i]) + bias_v, floor_v));
+                                }
+                            }
 #pragma unroll
                             for (int i = 0; i < 16; ++i) {
                                 out[i] = pack_bf16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
@@ -417,6 +435,10 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         } else {
                             tmem_ld32(t_addr + c * 32, out);
                             tmem_ld_wait();
+                            if (fuse) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) out[i] = __float_as_uint(fmaxf(__uint_as_float(out[i]) + bias_v, floor_v));
+                            }
                         }
                         store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0, slot);
                     }
@@ -788,7 +810,7 @@ bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int 
 
 cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
                            const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
-                           int nt_override, const ConvGeom *conv, cudaStream_t st) {
+                           int nt_override, const ConvGeom *conv, const Epilogue &epilogue, cudaStream_t st) {
     const TcImageLayout L = tc_image_layout(g, sparse);
     static int sm_count = 0;
     if (!sm_count) {
@@ -841,6 +863,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.walk_col = reinterpret_cast<const int32_t *>(d_exec + L.walk_col_off);
     p.walk_len = reinterpret_cast<const int32_t *>(d_exec + L.walk_len_off);
     p.status = d_status;
+    p.bias = epilogue.bias; p.relu = epilogue.relu;
     p.nst = L.nst; p.wcap = L.wcap; p.bk = g.bk; p.rows = g.rows; p.ncols = ncols; p.y = d_y; p.ldy = ldy;
     p.n_col_tiles = (int)((ncols + nt * kBoxN - 1) / (nt * kBoxN));
     if (conv) p.n_col_tiles = p.cv_tiles_x * p.cv_tiles_y * ((conv->batch + p.cv_tb - 1) / p.cv_tb);

@@ -62,3 +62,17 @@ def test_all_ones_kernel_counts_the_window():
     got = oracle.conv_fp64(np.ones((1, 18)), 3, 3, act, 1).reshape(4, 4)
     inside = np.array([[4, 6, 6, 4], [6, 9, 9, 6], [6, 9, 9, 6], [4, 6, 6, 4]]) * 2.0
     assert np.array_equal(got, inside)
+
+
+def test_layer_epilogue_hand_values():
+    # bias per row, then the rectifier: written out by hand
+    y = np.array([[1.5, -2.0, 0.0], [-0.25, 4.0, -4.0]])
+    b = np.array([0.5, -1.0], dtype=np.float32)
+    assert np.array_equal(oracle.bias_relu(y), y)
+    assert np.array_equal(oracle.bias_relu(y, b), [[2.0, -1.5, 0.5], [-1.25, 3.0, -5.0]])
+    assert np.array_equal(oracle.bias_relu(y, b, relu=True), [[2.0, 0.0, 0.5], [0.0, 3.0, 0.0]])
+    assert np.array_equal(oracle.bias_relu(y, None, relu=True), [[1.5, 0.0, 0.0], [0.0, 4.0, 0.0]])
+    # against numpy on a random case
+    rng = np.random.default_rng(0)
+    y = rng.standard_normal((7, 13)); b = rng.standard_normal(7).astype(np.float32)
+    np.testing.assert_array_equal(oracle.bias_relu(y, b, relu=True), np.maximum(y + b.astype(np.float64)[:, None], 0))
