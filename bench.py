@@ -339,6 +339,37 @@ def measure_conv(torch, B, dev, peaks, flush_l2, iters=9):
     return out
 
 
+def measure_saliency(torch, B, dev, peaks, flush_l2, shared, samples=4, iters=9):
+    """Saliency score of Eq. 1 on the sweep layer (4096 x 4096): `samples` gradient tensors (bf16) accumulated,
+    then S = |mean g * W|.  HBM roofline: per accumulate 2 + 4 (+ 4 after the first) bytes per weight, per
+    finish 4 + 2 + 4."""
+    _d_s, d_w, _d_x = shared
+    rows, k = d_w.shape
+    stream = torch.cuda.current_stream()
+    g = torch.Generator(device=dev); g.manual_seed(77)
+    grads = [(torch.randn((rows, k), device=dev, generator=g) * 1e-2).to(torch.bfloat16) for _ in range(samples)]
+    acc = torch.empty((rows, k), dtype=torch.float32, device=dev)
+    s = torch.empty((rows, k), dtype=torch.float32, device=dev)
+    ts = []
+    for i in range(3 + iters):
+        flush_l2()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for j, gr in enumerate(grads):
+            B.crisp_saliency_accumulate(gr, 0, k, rows, k, acc, k, j == 0)
+        B.crisp_saliency_finish(acc, k, d_w, k, rows, k, samples, s, k)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            ts.append(a.elapsed_time(b))
+    ms = float(np.mean(ts))
+    n = rows * k
+    alg = n * (6 + (samples - 1) * 10 + 10)
+    return {"workload": f"saliency_{rows}x{k}_{samples}samples_bf16grad", "us": ms * 1e3, "launches": samples + 1,
+            "algorithmic_bytes": int(alg), "achieved_gbs": alg / (ms * 1e-3) / 1e9,
+            "roofline_frac": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+
 def recorded_traffic(workload, kernel):
     """DRAM bytes per launch from the committed ncu capture, or None when the kernel source has
     changed since the counters were taken."""
@@ -527,6 +558,7 @@ def run_ours(args, layer, rank, world):
         out["cells"] = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
         out["global_rank"] = measure_global_rank(torch, B, dev, not args.no_cpu_baseline)
         out["conv"] = measure_conv(torch, B, dev, peaks, flush_l2)
+        out["saliency"] = measure_saliency(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)

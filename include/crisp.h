@@ -155,6 +155,24 @@ CRISP_API crisp_status_t crisp_build_mask_static(const float *d_saliency, int64_
                                                  void *stream, crisp_mask_t *out);
 
 /*
+ * Class-aware saliency score (Sec. III-C "Pruning Metric", Eq. 1): the first-order Taylor estimate
+ * T_w = | (1/H) * sum_i g_i (.) W | with the loss gradient g averaged over the H samples of the
+ * user's classes.  The gradients are the caller's (one tensor per sample or mini-batch):
+ *   crisp_saliency_accumulate   acc = g (first = 1) or acc += g (first = 0), fp32, in call order
+ *   crisp_saliency_finish       S = | acc * (1 / samples) * W |, fp32: the input of crisp_build_mask
+ * d_grad: [rows, k] bf16 (grad_dtype 0) or fp32 (1); d_acc, d_saliency: [rows, k] fp32; d_w_bf16:
+ * [rows, k] bf16; leading dimensions in elements.  Arithmetic is fp32 in exactly this order (sum of
+ * the samples in call order, times the rounded reciprocal of `samples`, times the weight), so the
+ * result does not depend on the launch shape.  Nothing is allocated.
+ */
+CRISP_API crisp_status_t crisp_saliency_accumulate(const void *d_grad, int32_t grad_dtype, int64_t ld_g,
+                                                   int32_t rows, int32_t k, float *d_acc, int64_t ld_acc,
+                                                   int32_t first, void *stream);
+CRISP_API crisp_status_t crisp_saliency_finish(const float *d_acc, int64_t ld_acc, const uint16_t *d_w_bf16,
+                                               int64_t ld_w, int32_t rows, int32_t k, int32_t samples,
+                                               float *d_saliency, int64_t ld_s, void *stream);
+
+/*
  * Global rank selection across the layers of a network: Algorithm 1 of the paper between the
  * block scores and the pruning itself (Sec. III-C, "Pruning Algorithm": sort the block scores
  * inside every row of the block grid, add the o-th smallest score of every row into the

@@ -234,3 +234,16 @@ def bias_relu(y: np.ndarray, bias=None, relu: bool = False) -> np.ndarray:
     if rc:
         raise ValueError(f"oracle_bias_relu rc={rc}")
     return out
+
+
+def saliency(grads: np.ndarray, w_bits: np.ndarray) -> np.ndarray:
+    """Eq. 1: |mean over samples of g  *  W|.  grads [H, rows, k] (any float), w_bits bf16 patterns -> fp64."""
+    g = np.ascontiguousarray(grads, dtype=np.float64)
+    w = np.ascontiguousarray(w_bits, dtype=np.uint16)
+    h, rows, k = g.shape
+    out = np.zeros((rows, k), dtype=np.float64)
+    rc = lib().oracle_saliency(_p(g, C.c_double), C.c_int(h), _p(w, C.c_uint16), C.c_int(rows), C.c_int(k),
+                               _p(out, C.c_double))
+    if rc:
+        raise ValueError(f"oracle_saliency rc={rc}")
+    return out

@@ -539,3 +539,23 @@ int oracle_bias_relu(double *y, int rows, int64_t ncols, const float *bias, int 
         }
     return 0;
 }
+
+/* ---------------------------------------------------------------- saliency score */
+
+/*
+ * Class-aware saliency score, Sec. III-C "Pruning Metric", Eq. 1:
+ *   T_w = | (1/H) * sum over the H samples of g_i  (.)  W |      (element-wise)
+ * grads: H tensors [rows, k] laid out one after the other, as doubles (the values the caller's
+ * gradients hold); w: bf16 bit patterns; out: fp64.
+ */
+int oracle_saliency(const double *grads, int samples, const uint16_t *w, int rows, int k, double *out)
+{
+    if (!grads || !w || !out || samples <= 0 || rows <= 0 || k <= 0) return -1;
+    const int64_t n = (int64_t)rows * k;
+    for (int64_t e = 0; e < n; ++e) {
+        double sum = 0.0;
+        for (int i = 0; i < samples; ++i) sum += grads[(int64_t)i * n + e];
+        out[e] = fabs(sum / (double)samples * bf16_to_double(w[e]));
+    }
+    return 0;
+}

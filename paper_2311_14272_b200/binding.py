@@ -80,6 +80,8 @@ def load(path: Optional[str] = None):
         "crisp_decode": [vp, vp, i64, vp],
         "crisp_spmm": [vp, vp, i64, i64, vp, i64, i32, vp],
         "crisp_spmm_conv": [vp, vp, P(ConvDesc), vp, i64, i32, vp],
+        "crisp_saliency_accumulate": [vp, i32, i64, i32, i32, vp, i64, i32, vp],
+        "crisp_saliency_finish": [vp, i64, vp, i64, i32, i32, i32, vp, i64, vp],
         "crisp_set_path": [vp, i32],
         "crisp_set_epilogue": [vp, vp, i32],
         "crisp_device_status": [vp, vp, P(i32)],
@@ -150,6 +152,18 @@ def crisp_mask_sizes(desc: LayerDesc):
     a, b = C.c_size_t(), C.c_size_t()
     _check(load().crisp_mask_sizes(C.byref(desc), C.byref(a), C.byref(b)), "crisp_mask_sizes")
     return a.value, b.value
+
+
+def crisp_saliency_accumulate(d_grad, grad_dtype: int, ld_g: int, rows: int, k: int, d_acc, ld_acc: int, first: bool,
+                              stream=None):
+    _check(load().crisp_saliency_accumulate(_ptr(d_grad), grad_dtype, ld_g, rows, k, _ptr(d_acc), ld_acc,
+                                            1 if first else 0, _stream(stream)), "crisp_saliency_accumulate")
+
+
+def crisp_saliency_finish(d_acc, ld_acc: int, d_w, ld_w: int, rows: int, k: int, samples: int, d_saliency, ld_s: int,
+                          stream=None):
+    _check(load().crisp_saliency_finish(_ptr(d_acc), ld_acc, _ptr(d_w), ld_w, rows, k, samples, _ptr(d_saliency), ld_s,
+                                        _stream(stream)), "crisp_saliency_finish")
 
 
 def crisp_mask_scores(desc: LayerDesc, d_workspace):

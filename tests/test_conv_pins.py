@@ -76,3 +76,20 @@ def test_layer_epilogue_hand_values():
     rng = np.random.default_rng(0)
     y = rng.standard_normal((7, 13)); b = rng.standard_normal(7).astype(np.float32)
     np.testing.assert_array_equal(oracle.bias_relu(y, b, relu=True), np.maximum(y + b.astype(np.float64)[:, None], 0))
+
+
+def test_saliency_score_hand_values_and_numpy():
+    # Eq. 1 on values small enough to do by hand: mean gradient times weight, magnitude
+    w = bf16(np.array([[2.0, -0.5, 4.0]]))
+    g = np.array([[[1.0, 2.0, -1.0]], [[3.0, -2.0, -3.0]]])          # means 2, 0, -2
+    assert np.array_equal(oracle.saliency(g, w), [[4.0, 0.0, 8.0]])
+    rng = np.random.default_rng(4)
+    g = rng.standard_normal((5, 6, 9))
+    wb = bf16(rng.standard_normal((6, 9)))
+    want = np.abs(g.mean(axis=0) * wl.bf16_bits_to_f32(wb).astype(np.float64))
+    np.testing.assert_allclose(oracle.saliency(g, wb), want, rtol=1e-14, atol=0)
+    # the three cases the paper lists keep their order: small*small < large*small ~ small*large < large*large
+    w2 = bf16(np.array([[0.01, 1.0, 0.01, 1.0]]))
+    g2 = np.array([[[0.01, 0.01, 1.0, 1.0]]])
+    s = oracle.saliency(g2, w2)[0]
+    assert s[0] < s[1] and s[0] < s[2] and s[1] < s[3] and s[2] < s[3]
