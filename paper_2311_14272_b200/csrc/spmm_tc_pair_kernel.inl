@@ -3,14 +3,62 @@
 // Shared memory per CTA (identical layout in both CTAs, 1024-byte aligned):
 //   num_stages x [weight tile | metadata (sparse) | 2 boxes of X (this CTA's 128 columns)]
 //   | 4 warps x 2 staging tiles | barriers | TMEM base | abort flag
+// The leader's MMA issuer loop with the number of MMAs per kept block fixed at compile time (the loop is
+// bound by this one thread's instruction latency: descriptors of stage 0 are built once, a later stage or
+// K step only moves the start-address field, and the MMAs of a block are a straight line).
+struct PairMmaArgs {
+    uint32_t ring, bar_full, bar_empty, bar_tfull, bar_tempty, tmem_base;
+    int first_pair_tile, pair_tile_stride;
+    volatile int *abort_flag;
+};
+template <bool kSparse, int NM>
+__device__ __forceinline__ void pair_mma_role(const PairParams &p, const PairMmaArgs &a) {
+    constexpr uint32_t kIdesc = make_idesc_pair(kSparse);
+    constexpr int kMetaCol = kPairTileN;          // two 4-column metadata buffers after the accumulator
+    const uint64_t a_desc0 = make_smem_desc(a.ring, 2048, 128, kLayoutNone);
+    const uint64_t b_desc0 = make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
+    const uint64_t m_desc0 = make_smem_desc(a.ring + p.a_bytes, 128, 128, kLayoutNone);
+    const uint32_t stage_step = p.stage_bytes >> 4, ring_span = p.num_stages * stage_step;
+    uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc_ph = 0, meta_buf = 0;
+    for (int t = a.first_pair_tile; t < p.num_tiles && !*a.abort_flag; t += a.pair_tile_stride) {
+        const int len = p.pair_len[t % p.npairs];
+        if (!mbar_wait(a.bar_tempty, acc_ph ^ 1u, a.abort_flag)) break;
+        tc_fence_after();
+        uint32_t accum = 0;
+        bool ok = true;
+        for (int e = 0; e < len; ++e) {
+            if (!mbar_wait(full, ph, a.abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t ad = a_desc0 + off, bd = b_desc0 + off;
+            if constexpr (kSparse) {
+                const uint32_t meta_tmem = a.tmem_base + kMetaCol + 4 * meta_buf;
+                tmem_copy_128x128b_pair(meta_tmem, m_desc0 + off);
+#pragma unroll
+                for (int j = 0; j < NM; ++j)
+                    mma_sparse_pair(a.tmem_base, ad + j * 256, bd + j * 256, kIdesc | (uint32_t)(j & 1), accum | (uint32_t)j,
+                                    meta_tmem + (j & ~1));
+                meta_buf ^= 1u;
+            } else {
+#pragma unroll
+                for (int j = 0; j < NM; ++j) mma_dense_pair(a.tmem_base, ad + j * 256, bd + j * 128, kIdesc, accum | (uint32_t)j);
+            }
+            accum = 1u;
+            mma_commit_pair(empty);                 // both CTAs may refill this stage
+            off += stage_step; full += 8; empty += 8;
+            if (off == ring_span) { off = 0; full = a.bar_full; empty = a.bar_empty; ph ^= 1u; }
+        }
+        if (!ok) break;
+        mma_commit_pair(a.bar_tfull);               // both CTAs' accumulators are complete
+        acc_ph ^= 1u;
+    }
+}
+
 template <bool kSparse, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 spmm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                     const __grid_constant__ CUtensorMap map_a, PairParams p) {
     constexpr int kTmemCols = 512;
-    constexpr int kMetaCol = kPairTileN;          // two 4-column metadata buffers after the accumulator
     constexpr int kOutCols = 128 / (int)sizeof(OutT);
-    constexpr uint32_t kIdesc = make_idesc_pair(kSparse);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -48,39 +96,44 @@ spmm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 
     if (warp == 0) {
         // ------------------------------------------------ producer (both CTAs): step 1
+        // (running stage/barrier addresses and image rows: this thread's own instruction latency bounds the loop)
         if (lane == 0) {
-            const uint32_t leader_full = map_to_cta(bar_full, 0);
-            uint32_t s = 0, ph = 0;
+            constexpr int kAhead = 8;            // union-list entries held in registers ahead of their use
+            const uint32_t leader_full0 = map_to_cta(bar_full, 0);
+            const uint32_t ring_end = ring + p.num_stages * p.stage_bytes;
+            const int entry_rows = (int)(p.entry_bytes >> 8);
+            uint32_t dst = ring, full_own = bar_full, full_leader = leader_full0, empty = bar_empty, ph = 0;
             for (int t = first_pair_tile; t < p.num_tiles && !*abort_flag; t += pair_tile_stride) {
                 const int pr = t % p.npairs, ct = t / p.npairs;
                 const int st = 2 * pr + (int)rank;
                 const int len = p.pair_len[pr];
                 const int32_t *cols = p.pair_col + (int64_t)pr * p.pwcap;
                 const int32_t *src = p.pair_src + (int64_t)pr * p.pwcap * 2 + rank;
-                // list entries are global loads in this thread's serial loop: keep the next four in registers
-                int col_q[4], src_q[4];
+                const int base_row = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
+                const int xz = ct * 4 + kPairBoxes * (int)rank;
+                int col_q[kAhead], src_q[kAhead];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kAhead; ++u) {
                     col_q[u] = u < len ? __ldg(cols + u) : 0;
                     src_q[u] = u < len ? __ldg(src + 2 * u) : -1;
                 }
                 bool ok = true;
-                for (int e0 = 0; e0 < len && ok; e0 += 4) {
+                for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < kAhead; ++u) {
                         const int e = e0 + u;
                         if (e >= len) break;
                         const int krow = col_q[u] * p.bk;
                         const int idx = src_q[u];
-                        if (e + 4 < len) { col_q[u] = __ldg(cols + e + 4); src_q[u] = __ldg(src + 2 * (e + 4)); }
-                        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-                        const uint32_t dst = ring + s * p.stage_bytes;
-                        if (leader) mbar_expect_tx(bar_full + 8 * s, 2 * stage_tx);
-                        const int arow = idx >= 0 ? (int)((((int64_t)st * p.wcap + idx) * p.entry_bytes) >> 8) : p.image_rows;
-                        tma_load_2d_pair(dst, &map_a, 0, arow, leader_full + 8 * s);
-                        tma_load_3d_pair(dst + p.entry_bytes, &map_x, 0, krow, ct * 4 + kPairBoxes * (int)rank,
-                                         leader_full + 8 * s);
-                        if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                        if (e + kAhead < len) { col_q[u] = __ldg(cols + e + kAhead); src_q[u] = __ldg(src + 2 * (e + kAhead)); }
+                        if (!mbar_wait(empty, ph ^ 1u, abort_flag)) { ok = false; break; }
+                        if (leader) mbar_expect_tx(full_own, 2 * stage_tx);
+                        // a side that does not keep this block of the union loads a zero tile (row past the image)
+                        const int arow = idx >= 0 ? base_row + idx * entry_rows : p.image_rows;
+                        tma_load_2d_pair(dst, &map_a, 0, arow, full_leader);
+                        tma_load_3d_pair(dst + p.entry_bytes, &map_x, 0, krow, xz, full_leader);
+                        dst += p.stage_bytes; full_own += 8; full_leader += 8; empty += 8;
+                        if (dst == ring_end) { dst = ring; full_own = bar_full; full_leader = leader_full0; empty = bar_empty; ph ^= 1u; }
                     }
                 }
                 if (!ok) break;
@@ -89,40 +142,23 @@ spmm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (leader CTA only): steps 2 + 3
         if (leader && lane == 0) {
-            uint32_t s = 0, ph = 0, acc_ph = 0, meta_buf = 0;
-            for (int t = first_pair_tile; t < p.num_tiles && !*abort_flag; t += pair_tile_stride) {
-                const int len = p.pair_len[t % p.npairs];
-                if (!mbar_wait(bar_tempty, acc_ph ^ 1u, abort_flag)) break;
-                tc_fence_after();
-                bool ok = true;
-                for (int e = 0; e < len; ++e) {
-                    if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_smem = ring + s * p.stage_bytes;
-                    const uint32_t x_smem = a_smem + p.entry_bytes;
-                    if constexpr (kSparse) {
-                        const uint32_t meta_tmem = tmem_base + kMetaCol + 4 * meta_buf;
-                        tmem_copy_128x128b_pair(meta_tmem, make_smem_desc(a_smem + p.a_bytes, 128, 128, kLayoutNone));
-                        for (int j = 0; j < p.bk / 32; ++j) {
-                            const uint64_t ad = make_smem_desc(a_smem + j * 4096, 2048, 128, kLayoutNone);
-                            const uint64_t bd = make_smem_desc(x_smem + j * 4096, p.box_bytes, 1024, kLayoutSw128);
-                            mma_sparse_pair(tmem_base, ad, bd, kIdesc | (uint32_t)(j & 1), (e | j) ? 1u : 0u,
-                                            meta_tmem + (j & ~1));
-                        }
-                        meta_buf ^= 1u;
-                    } else {
-                        for (int j = 0; j < p.bk / 16; ++j) {
-                            const uint64_t ad = make_smem_desc(a_smem + j * 4096, 2048, 128, kLayoutNone);
-                            const uint64_t bd = make_smem_desc(x_smem + j * 2048, p.box_bytes, 1024, kLayoutSw128);
-                            mma_dense_pair(tmem_base, ad, bd, kIdesc, (e | j) ? 1u : 0u);
-                        }
-                    }
-                    mma_commit_pair(bar_empty + 8 * s);     // both CTAs may refill this stage
-                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+            const PairMmaArgs a{ring, bar_full, bar_empty, bar_tfull, bar_tempty, tmem_base, first_pair_tile,
+                                pair_tile_stride, abort_flag};
+            const int nmma = kSparse ? p.bk / 32 : p.bk / 16;
+            if constexpr (kSparse) {
+                switch (nmma) {
+                    case 1: pair_mma_role<true, 1>(p, a); break;
+                    case 2: pair_mma_role<true, 2>(p, a); break;
+                    case 3: pair_mma_role<true, 3>(p, a); break;
+                    default: pair_mma_role<true, 4>(p, a); break;
                 }
-                if (!ok) break;
-                mma_commit_pair(bar_tfull);                 // both CTAs' accumulators are complete
-                acc_ph ^= 1u;
+            } else {
+                switch (nmma) {
+                    case 2: pair_mma_role<false, 2>(p, a); break;
+                    case 4: pair_mma_role<false, 4>(p, a); break;
+                    case 6: pair_mma_role<false, 6>(p, a); break;
+                    default: pair_mma_role<false, 8>(p, a); break;
+                }
             }
         }
     } else {
