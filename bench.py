@@ -482,7 +482,11 @@ def run_ours(args, layer, rank, world):
             t_dense.append(a.elapsed_time(b))
     t_dense = np.array(t_dense)
 
-    # ---- end to end: pinned host inputs -> device, whole path, result back to pinned host memory
+    # ---- end to end: pinned host inputs -> device, whole path, result back to pinned host memory.
+    # Every step copies its own S, W and X from pinned host memory and its Y back; two sets of device
+    # buffers and two copy streams let the copies of step i+1 run while step i computes and reads back
+    # (PCIe is full duplex), as a caller that streams layers through the library would do.  The same
+    # loop on one stream (no overlap) is reported beside it.
     def e2e_step():
         d_s.copy_(h_s, non_blocking=True)
         d_w.view(torch.int16).copy_(h_w, non_blocking=True)
@@ -490,16 +494,59 @@ def run_ours(args, layer, rank, world):
         step()
         h_y.copy_(d_y, non_blocking=True)
 
+    d_in = [(d_s, d_w, d_x), (torch.empty_like(d_s), torch.empty_like(d_w), torch.empty_like(d_x))]
+    d_out = [d_y, torch.empty_like(d_y)]
+    h_out = [h_y, torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16).pin_memory()]
+    s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_cmp = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
+
+    def e2e_pipelined(n, start_event):
+        s_in.wait_event(start_event)
+        for it in range(n):
+            k = it & 1
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_cmp[k])               # the step that last read this buffer set is done
+                d_in[k][0].copy_(h_s, non_blocking=True)
+                d_in[k][1].view(torch.int16).copy_(h_w, non_blocking=True)
+                d_in[k][2].view(torch.int16).copy_(h_x, non_blocking=True)
+                ev_in[k].record(s_in)
+            stream.wait_event(ev_in[k])
+            stream.wait_event(ev_out[k])                 # this Y buffer has been read back
+            L.build_mask(d_in[k][0])
+            L.encode(d_in[k][1])
+            L.spmm(d_in[k][2], y=d_out[k])
+            ev_cmp[k].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_cmp[k])
+                h_out[k].copy_(d_out[k], non_blocking=True)
+                ev_out[k].record(s_out)
+        stream.wait_event(ev_out[0])
+        stream.wait_event(ev_out[1])
+
+    e2e_steps = max(3, min(args.steps, 10))
     for _ in range(2):
         e2e_step()
     barrier()
-    e2e_steps = max(3, min(args.steps, 10))
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
     b.record(stream)
     barrier()
+    e2e_serial_ms = a.elapsed_time(b) / e2e_steps
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    e2e_pipelined(2, a)
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    e2e_pipelined(e2e_steps, a)
+    b.record(stream)
+    barrier()
+    if not torch.equal(h_out[0], h_out[1]):
+        raise SystemExit("end-to-end pipeline: the two result buffers differ")
     e2e_ms = torch.tensor([a.elapsed_time(b) / e2e_steps], device=dev, dtype=torch.float64)
     if world > 1:
         dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
@@ -548,7 +595,8 @@ def run_ours(args, layer, rank, world):
                       "step": "crisp_build_mask + crisp_encode + crisp_spmm",
                       "l2": "flushed between steps (256 MiB overwritten, then read back, outside the event pairs)",
                       "parallelism": "replicas only" if world > 1 else "single GPU"},
-           "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
+           "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "serial_ms_per_step": e2e_serial_ms,
+                   "overlap": "copies of step i+1 overlap compute and read-back of step i (2 buffer sets, 3 streams)",
                    "h2d_bytes_per_step": int(h_s.numel() * 4 + h_w.numel() * 2 + h_x.numel() * 2),
                    "d2h_bytes_per_step": int(h_y.numel() * 2)},
            "gpu_launches": sum(kernels_per_step.values()) * args.steps, "kernels_per_step": kernels_per_step,
