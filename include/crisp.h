@@ -287,9 +287,10 @@ CRISP_API crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, 
  *               ho = height + 2*pad - kernel_h + 1, wo likewise
  * The handle's k must equal kernel_h*kernel_w*channels (BAD_SHAPE otherwise).  Supported
  * (UNSUPPORTED otherwise; lower the convolution to a matrix and call crisp_spmm): block_k = 64,
- * channels a multiple of 64, wo*sizeof(Y element) and ldy*sizeof(Y element) multiples of 16
- * bytes, a tensor-core execution image and at least one kept block.  Same tolerance and status
- * reporting as crisp_spmm.
+ * channels a multiple of 64, a tensor-core execution image and at least one kept block.  Y is
+ * written by bulk tensor stores when d_y is 16-byte aligned and wo*sizeof(Y element) and
+ * ldy*sizeof(Y element) are multiples of 16 bytes, element by element otherwise (e.g. 28- or
+ * 14-pixel rows of bf16).  Same tolerance and status reporting as crisp_spmm.
  */
 typedef struct {
     int32_t batch, height, width, channels;   /* input activation, NHWC                         */

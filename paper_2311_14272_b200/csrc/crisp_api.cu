@@ -283,8 +283,8 @@ crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, con
     const int es = y_dtype ? 4 : 2;
     // the gather needs whole k-blocks inside one filter tap, 128-byte channel slabs, and TMA-addressable tensors
     if (h->g.bk != 64 || cd->channels % h->g.bk != 0) return CRISP_UNSUPPORTED;
-    if (((int64_t)cg.wo * es) % 16 != 0 || (ldy * es) % 16 != 0 || !aligned(d_act_nhwc, 16) || !aligned(d_y, 16))
-        return CRISP_UNSUPPORTED;
+    if (!aligned(d_act_nhwc, 16)) return CRISP_UNSUPPORTED;
+    if (!aligned(d_y, es)) return CRISP_INVALID_ARG;
     const int path = h->forced_path >= 0 ? h->forced_path : h->exec_kind;
     if (path == CRISP_PATH_DIRECT || h->g.kkeep == 0) return CRISP_UNSUPPORTED;
     const char *nt = std::getenv("CRISP_TC_NT");

@@ -48,6 +48,9 @@ struct TcParams {
     int cv_cpt;                 // k-blocks per filter tap = channels / bk
     int cv_kw, cv_pad;          // filter width, zero padding
     int cv_wo, cv_ho, cv_batch; // output width, height, images
+    int cv_plain;               // Y rows are not TMA-addressable (wo * element size not a multiple of 16 bytes):
+                                // the epilogue stores element by element
+    int cv_tw_log2, cv_img_log2;   // log2(tw), log2(tw * th)
     const float *bias;          // layer epilogue: Y = act(W*X + bias); nullptr = no bias
     int relu;
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
@@ -90,6 +93,28 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         const int img = col0 / per_image;
         cx = org.x; cy = org.y + (col0 - img * per_image) / p.cv_tw; cb = org.b + img;
         inside = cx < p.cv_wo && cy < p.cv_ho && cb < p.cv_batch;
+    }
+    if constexpr (kConv) {
+        if (p.cv_plain) {
+            // every lane writes the kOutCols pixels of its row one by one: pixel c of the chunk is
+            // (image, y, x) = box order inside the tile, clipped at the image borders
+            const int row = y0 + lane;
+            if (row < p.rows) {
+                OutT *yrow = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy;
+#pragma unroll
+                for (int c = 0; c < kOutCols; ++c) {
+                    const int col = col0 + c;
+                    const int img = col >> p.cv_img_log2, rem = col & ((1 << p.cv_img_log2) - 1);
+                    const int gy = org.y + (rem >> p.cv_tw_log2), gx = org.x + (rem & (p.cv_tw - 1)), gb = org.b + img;
+                    if (gx < p.cv_wo && gy < p.cv_ho && gb < p.cv_batch) {
+                        OutT *dst = yrow + ((int64_t)gb * p.cv_ho + gy) * p.cv_wo + gx;
+                        if constexpr (sizeof(OutT) == 2) *dst = (OutT)((out[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
+                        else *dst = __uint_as_float(out[c]);
+                    }
+                }
+            }
+            return;
+        }
     }
     if (!kConv && x0 + kOutCols > p.ncols && (p.ncols * (int64_t)sizeof(OutT)) % 16 != 0) {
         const int row = y0 + lane;
@@ -244,7 +269,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_a);
-        prefetch_tensormap(&map_y);
+        if (!(kConv && p.cv_plain)) prefetch_tensormap(&map_y);
     }
     if (p.walk_cache) {
         for (int i = threadIdx.x; i < p.nst; i += blockDim.x) s_walk[i] = p.walk_len[i];
@@ -903,6 +928,10 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.stg_swz_mask = 7;
     if (conv) {
         p.stg_swz_mask = (uint32_t)(p.cv_tw * (f32 ? 4 : 2)) / 16 - 1;      // 128 / 64 / 32 / 16-byte inner box of map_y
+        p.cv_plain = ((int64_t)conv->wo * (f32 ? 4 : 2)) % 16 != 0 || (ldy * (f32 ? 4 : 2)) % 16 != 0 ||
+                     reinterpret_cast<uintptr_t>(d_y) % 16 != 0;
+        for (p.cv_tw_log2 = 0; (1 << p.cv_tw_log2) < p.cv_tw; ++p.cv_tw_log2) {}
+        for (p.cv_img_log2 = 0; (1 << p.cv_img_log2) < p.cv_tw * p.cv_th; ++p.cv_img_log2) {}
         // activation [batch][height][width][channels] and Y [rows][batch][ho][wo] as 4-D tensors
         if (!p.a_map) return cudaErrorInvalidValue;
         p.x_map_3d = 0;
@@ -913,7 +942,8 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
         const uint64_t es = f32 ? 4 : 2, wo = (uint64_t)conv->wo, ho = (uint64_t)conv->ho;
         const uint64_t yd[4] = {wo, ho, (uint64_t)conv->batch, (uint64_t)g.rows}, ys[3] = {wo * es, ho * wo * es, (uint64_t)ldy * es};
         const uint32_t yb[4] = {(uint32_t)p.cv_tw, (uint32_t)((f32 ? 32 : 64) / p.cv_tw), 1u, p.stg_tile_bytes / 128};
-        if (!make_map_4d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (int)es, d_y, yd, ys, yb))
+        if (p.cv_plain) my = CUtensorMap{};
+        else if (!make_map_4d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (int)es, d_y, yd, ys, yb))
             return cudaErrorInvalidValue;
     } else {
         p.x_map_3d = (ncols % kBoxN == 0) &&

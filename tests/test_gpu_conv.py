@@ -40,6 +40,9 @@ CASES = [
     (128, 1, 1, 0, 192, 2, 8, 16, 2, 8, 64, 0.67),        # pointwise
     (64, 5, 3, 1, 64, 2, 12, 16, 3, 4, 64, 0.6),          # dense-tile image (3:4), output shorter than input
     (160, 3, 3, 0, 64, 1, 18, 34, 4, 8, 32, 0.75),        # no padding: 16 x 32 outputs from 18 x 34
+    (96, 3, 3, 1, 64, 3, 14, 14, 2, 4, 64, 0.5),          # 14-pixel rows: Y is stored element by element
+    (128, 3, 3, 1, 128, 2, 28, 28, 1, 4, 64, 0.25),       # 28-pixel rows, two k-blocks per tap
+    (64, 3, 3, 1, 64, 2, 9, 11, 3, 4, 32, 0.8),           # odd sizes in both directions, dense-tile image
 ]
 
 
@@ -94,8 +97,6 @@ def test_unsupported_shapes_are_refused(env):
     B, torch = env
     wt, sal, act = conv_inputs(64, 3, 3, 64, 1, 8, 14, seed=1)
     L = gpu_layer(B, torch, wt, sal, 2, 4, 64, 64, 0.5)
-    with pytest.raises(B.CrispError):          # 14 outputs per row: 28 bytes, not addressable by TMA
-        L.spmm_conv(bf16_dev(act, torch), 3, 3, 1)
     with pytest.raises(B.CrispError):          # the handle's k is 9 * 64, not 9 * 32
         L.spmm_conv(bf16_dev(act[..., :32].copy(), torch), 3, 3, 1)
     wt2, sal2, act2 = conv_inputs(64, 3, 3, 32, 1, 8, 16, seed=2)
