@@ -96,20 +96,45 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
     }
     if constexpr (kConv) {
         if (p.cv_plain) {
-            // every lane writes the kOutCols pixels of its row one by one: pixel c of the chunk is
-            // (image, y, x) = box order inside the tile, clipped at the image borders
-            const int row = y0 + lane;
-            if (row < p.rows) {
-                OutT *yrow = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy;
+            // Through the warp's staging tile, so that a store instruction covers consecutive pixels of one
+            // row of W: lane r writes its row (swizzled 16-byte chunks), then for every row the lanes take the
+            // chunk's pixels side by side.  Pixel c of the chunk is (image, y, x) in box order inside the tile,
+            // clipped at the image borders.
+            constexpr int kPer = kOutCols / 32;          // pixels per lane and row
+            int64_t pix_off[kPer];
+            uint32_t smem_off[kPer];
+            bool pix_ok[kPer];
 #pragma unroll
-                for (int c = 0; c < kOutCols; ++c) {
-                    const int col = col0 + c;
-                    const int img = col >> p.cv_img_log2, rem = col & ((1 << p.cv_img_log2) - 1);
-                    const int gy = org.y + (rem >> p.cv_tw_log2), gx = org.x + (rem & (p.cv_tw - 1)), gb = org.b + img;
-                    if (gx < p.cv_wo && gy < p.cv_ho && gb < p.cv_batch) {
-                        OutT *dst = yrow + ((int64_t)gb * p.cv_ho + gy) * p.cv_wo + gx;
-                        if constexpr (sizeof(OutT) == 2) *dst = (OutT)((out[c >> 1] >> (16 * (c & 1))) & 0xFFFFu);
-                        else *dst = __uint_as_float(out[c]);
+            for (int t = 0; t < kPer; ++t) {
+                const int c = lane + 32 * t, col = col0 + c;
+                const int img = col >> p.cv_img_log2, rem = col & ((1 << p.cv_img_log2) - 1);
+                const int gy = org.y + (rem >> p.cv_tw_log2), gx = org.x + (rem & (p.cv_tw - 1)), gb = org.b + img;
+                pix_ok[t] = gx < p.cv_wo && gy < p.cv_ho && gb < p.cv_batch;
+                pix_off[t] = ((int64_t)gb * p.cv_ho + gy) * p.cv_wo + gx;
+                smem_off[t] = (uint32_t)c * sizeof(OutT);
+            }
+            const int rpp = (int)(p.stg_tile_bytes / 128);      // rows per pass: 16 or 32
+            for (int h = 0; h < 32 / rpp; ++h) {
+                if (y0 + rpp * h >= p.rows) break;
+                __syncwarp();
+                if (lane / rpp == h) {
+                    uint8_t *tile = stg_gen + (lane % rpp) * 128;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(tile + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                }
+                __syncwarp();
+                for (int r = 0; r < rpp; ++r) {
+                    const int row = y0 + rpp * h + r;
+                    if (row >= p.rows) break;
+                    OutT *yrow = reinterpret_cast<OutT *>(p.y) + (int64_t)row * p.ldy;
+                    const uint8_t *trow = stg_gen + r * 128;
+#pragma unroll
+                    for (int t = 0; t < kPer; ++t) {
+                        const uint32_t chunk = (smem_off[t] >> 4) ^ (uint32_t)((rpp * h + r) & 7);
+                        const OutT v = *reinterpret_cast<const OutT *>(trow + (chunk << 4) + (smem_off[t] & 15u));
+                        if (pix_ok[t]) yrow[pix_off[t]] = v;
                     }
                 }
             }
