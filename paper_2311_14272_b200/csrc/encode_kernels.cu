@@ -63,13 +63,22 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
     if (threadIdx.x == 0) blk_col[blk] = jb;
     __syncthreads();
 
-    for (int item = threadIdx.x; item < g.bm * groups; item += blockDim.x) {
-        const int r = item / groups, gi = item - r * groups;
-        const int64_t row = (int64_t)rt * g.bm + r;
-        const int64_t col0 = (int64_t)jb * g.bk + (int64_t)gi * M;
-        uint16_t v[M];
-        load_group<M>(w, ld, g.rows, g.k, row, col0, vec_ok, v);
-        uint32_t bits = (nm_bits[row * g.wpr + (col0 >> 5)] >> (col0 & 31)) & ((1u << M) - 1u);
+    // a thread takes eight consecutive elements of a row (one 16-byte load: two groups of 4 or one of 8)
+    constexpr int kGroupsPerLoad = 8 / M;
+    const int loads_per_row = g.bk / 8;
+    for (int li = threadIdx.x; li < g.bm * loads_per_row; li += blockDim.x) {
+      const int r = li / loads_per_row, c8 = li - r * loads_per_row;
+      const int64_t row = (int64_t)rt * g.bm + r;
+      const int64_t col8 = (int64_t)jb * g.bk + (int64_t)c8 * 8;
+      uint16_t v8[8];
+      load_group<8>(w, ld, g.rows, g.k, row, col8, vec_ok, v8);
+      const uint32_t bits8 = (nm_bits[row * g.wpr + (col8 >> 5)] >> (col8 & 31)) & 0xFFu;
+#pragma unroll
+      for (int sub = 0; sub < kGroupsPerLoad; ++sub) {
+        const int gi = c8 * kGroupsPerLoad + sub;
+        const int item = r * groups + gi;
+        const uint16_t *v = v8 + sub * M;
+        const uint32_t bits = (bits8 >> (sub * M)) & ((1u << M) - 1u);
         if constexpr (TILE == CRISP_PATH_DENSE) {
 #pragma unroll
             for (int t = 0; t < M; ++t)
@@ -118,6 +127,7 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
             atomicOr(&s_idx[bit0 >> 5], field << sh);
             if (sh + kIdxBits * cnt > 32) atomicOr(&s_idx[(bit0 >> 5) + 1], field >> (32 - sh));
         }
+      }
     }
     __syncthreads();
     // vals_per_block is a multiple of 32 values = 64 bytes, the block's slice starts 64-byte aligned
@@ -170,8 +180,8 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
     const size_t vpb = (size_t)g.vals_per_block();
     size_t smem = (vpb * g.idx_bits / 32) * sizeof(uint32_t) + (vpb + 7) / 8 * 16 + 16;
     if (tile_kind != 0) smem += entry_bytes;
-    // vector loads of a whole group need the group start aligned to its size in every row
-    const size_t gbytes = (size_t)g.m * 2;
+    // the 16-byte loads of eight elements need every row to start 16-byte aligned (block columns are multiples of 32)
+    const size_t gbytes = 16;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(d_w) % gbytes == 0) && ((size_t)ld * 2 % gbytes == 0);
 #define CRISP_ENCODE_LAUNCH(MV, TV)                                                                          \
     do {                                                                                                     \
