@@ -79,6 +79,7 @@ struct TcImageLayout {
     int r;                  // row tiles per 128-row CTA tile
     int nst;                // 128-row CTA tiles
     int wcap;               // capacity of one CTA tile's walk list (union of its row tiles' kept blocks)
+    int stack;              // copies of the image, each shifted by 128 / stack rows (thin single-tile layers)
     uint32_t a_bytes;       // weight tile bytes per walk entry
     uint32_t entry_bytes;   // weight tile + metadata
     size_t walk_col_off, walk_len_off, image_off, total_bytes;   // offsets inside the exec payload

@@ -51,6 +51,10 @@ struct TcParams {
     int cv_plain;               // Y rows are not TMA-addressable (wo * element size not a multiple of 16 bytes):
                                 // the epilogue stores element by element
     int cv_tw_log2, cv_img_log2;   // log2(tw), log2(tw * th)
+    // Thin layers (one CTA tile, at most 128 / stack rows; matrix mode): a tile covers `stack` column tiles, one per
+    // group of 128 / stack accumulator lanes.  For group q the walk is run again with the image copy whose weights
+    // sit in that group's rows (all other rows zero) against the X columns of column tile ct * stack + q.
+    int stack;
     const float *bias;          // layer epilogue: Y = act(W*X + bias); nullptr = no bias
     int relu;
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
@@ -215,7 +219,7 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
     const uint32_t stage_step = p.stage_bytes >> 4, ring_span = p.num_stages * stage_step;
     uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
     for (int t = blockIdx.x; t < p.num_tiles && !*a.abort_flag; t += gridDim.x) {
-        const int len = a.walk_len[t % p.nst];
+        const int len = a.walk_len[t % p.nst] * p.stack;
         if (!mbar_wait(a.bar_tempty + 8 * acc, acc_ph ^ 1u, a.abort_flag)) break;
         tc_fence_after();
         const uint32_t d_tmem = a.tmem_base + acc * kTileN;
@@ -329,13 +333,16 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int32_t *cols = walk_col + (int64_t)st * p.wcap;
                 const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
                 const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
-                int arow = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
+                int arow0 = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
                 // The block column of entry e is a load in this thread's serial loop; left where it is used
                 // it costs a round trip per stage.  Keep the next kAhead in registers.
+                bool ok = true;
+              for (int q = 0; q < p.stack && ok; ++q) {
+                int arow = arow0 + q * p.wcap * (int)entry_rows;      // image copy q (stack > 1 only with one CTA tile)
+                const int xbox = (ct * p.stack + q) * NT;             // first 64-column box of this group's X columns
                 int col_q[kAhead];
 #pragma unroll
                 for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
-                bool ok = true;
                 for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
@@ -358,25 +365,26 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             // tiled loads pipeline (untiled bulk copies are served one at a time): the weight
                             // tile comes in as a box of 256-byte image rows, the NT boxes of X as one 3-D load
                             tma_load_2d(dst, &map_a, 0, arow, full);
-                            tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, full);
+                            tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, xbox, full);
                             arow += (int)entry_rows;
                         } else {
                             if (p.a_map)
-                                tma_load_2d(dst, &map_a, 0, (int)((((int64_t)st * p.wcap + e) * p.entry_bytes) >> 8), full);
+                                tma_load_2d(dst, &map_a, 0, arow + e * (int)entry_rows, full);
                             else
-                                bulk_load(dst, img + (int64_t)e * p.entry_bytes, p.entry_bytes, full);
+                                bulk_load(dst, img + ((int64_t)q * p.wcap + e) * p.entry_bytes, p.entry_bytes, full);
                             if (p.x_map_3d) {
-                                tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, ct * NT, full);
+                                tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, xbox, full);
                             } else {
 #pragma unroll
                                 for (int b = 0; b < NT; ++b)
-                                    tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, ct * kTileN + b * kBoxN, krow, full);
+                                    tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, (xbox + b) * kBoxN, krow, full);
                             }
                         }
                         dst += p.stage_bytes; full += 8; empty += 8;
                         if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
                     }
                 }
+              }
                 if (!ok) break;
             }
         }
@@ -422,8 +430,13 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             if (!go) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + acc * kTileN + ((uint32_t)(32 * q) << 16);
-            const int y0 = st * kTileM + 32 * q;
-            const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
+            // lane quarter q holds rows 32q.. of the CTA tile; in a stacked tile it belongs to column-tile group
+            // 32q / (128 / stack) and holds rows (32q) mod (128 / stack) of W
+            // (stack is 1, 2 or 4: 32q / (128 / stack) = q * stack / 4)
+            const int grp = (q * p.stack) >> 2;
+            const int y0 = st * kTileM + 32 * q - grp * (kTileM >> (p.stack >> 1));
+            TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
+            if constexpr (!kConv) org.x = (ct * p.stack + grp) * kTileN;
             // layer epilogue on the fp32 accumulator: this lane's row gets its bias, then the activation
             const bool fuse = p.bias != nullptr || p.relu != 0;
             const float bias_v = (p.bias != nullptr && y0 + lane < p.rows) ? p.bias[y0 + lane] : 0.f;
@@ -589,13 +602,18 @@ build_walks_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int n
 template <bool kSparse>
 __global__ void __launch_bounds__(256)
 build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16_t *__restrict__ vals,
-                   const uint32_t *__restrict__ idx, int r, int wcap, const int32_t *__restrict__ walk_col,
-                   const int32_t *__restrict__ walk_len, uint32_t a_bytes, uint32_t entry_bytes,
-                   uint8_t *__restrict__ image) {
+                   const uint32_t *__restrict__ idx, int r, int nst, int wcap, int stack,
+                   const int32_t *__restrict__ walk_col, const int32_t *__restrict__ walk_len, uint32_t a_bytes,
+                   uint32_t entry_bytes, uint8_t *__restrict__ image) {
     extern __shared__ uint4 s_tile4[];
     uint8_t *tile = reinterpret_cast<uint8_t *>(s_tile4);
     __shared__ int s_blk[4];
-    const int st = blockIdx.x / wcap, e = blockIdx.x - st * wcap;
+    // image entries are ordered [copy][CTA tile][walk entry]; copy q of a stacked layer (one CTA tile of at most
+    // 128 / stack rows) holds the same weights shifted down by q * 128 / stack rows
+    const int per_copy = nst * wcap;
+    const int copy = blockIdx.x / per_copy, in_copy = blockIdx.x - copy * per_copy;
+    const int st = in_copy / wcap, e = in_copy - st * wcap;
+    const int shift = copy * (kTileM / stack);
     if (e >= walk_len[st]) return;
     const int jb = walk_col[(int64_t)st * wcap + e];
     for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) s_tile4[i] = make_uint4(0, 0, 0, 0);
@@ -626,7 +644,7 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
     for (int sub = 0; sub < r; ++sub) {
         const int blk = s_blk[sub];
         if (blk < 0) continue;
-        const int row0 = sub * g.bm;
+        const int row0 = shift + sub * g.bm;
         __syncthreads();
         {
             const uint4 *vsrc = reinterpret_cast<const uint4 *>(vals + (int64_t)blk * vpb);      // vpb*2 is a multiple of 64
@@ -681,20 +699,20 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
         }
     }
     if constexpr (kSparse) {
-        // row tiles that do not keep this block still need valid (distinct, ascending) index pairs
+        // rows that carry no kept block here (row tiles that do not keep it, rows outside a stacked copy's
+        // window) still need valid (distinct, ascending) index pairs
         uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
-        for (int sub = 0; sub < r; ++sub) {
-            if (s_blk[sub] >= 0) continue;
-            for (int item = threadIdx.x; item < g.bm * (g.bk / 4); item += blockDim.x) {
-                const int lr = item / (g.bk / 4), qd = item - lr * (g.bk / 4);
-                const int row = sub * g.bm + lr, k0 = qd * 4;
-                const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
-                atomicOr(&meta[lrow * 4 + (k0 >> 5)], 0x4u << ((k0 & 15) + 16 * ((row >> 3) & 1)));
-            }
+        for (int item = threadIdx.x; item < kTileM * (g.bk / 4); item += blockDim.x) {
+            const int row = item / (g.bk / 4), qd = item - row * (g.bk / 4);
+            const int sub = row >= shift ? (row - shift) / g.bm : r;
+            if (sub < r && s_blk[sub] >= 0) continue;
+            const int k0 = qd * 4;
+            const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
+            atomicOr(&meta[lrow * 4 + (k0 >> 5)], 0x4u << ((k0 & 15) + 16 * ((row >> 3) & 1)));
         }
     }
     __syncthreads();
-    uint4 *out = reinterpret_cast<uint4 *>(image + ((int64_t)st * wcap + e) * entry_bytes);
+    uint4 *out = reinterpret_cast<uint4 *>(image + (int64_t)blockIdx.x * entry_bytes);      // [copy][st][e]
     for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = s_tile4[i];
 }
 
@@ -807,6 +825,10 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
     L.nst = (g.nrt + L.r - 1) / L.r;
     const int64_t cap = (int64_t)L.r * g.kkeep;
     L.wcap = (int)(cap < g.nblk ? cap : g.nblk);
+    // thin layers (a single CTA tile with at most 64 or 32 rows): 2 or 4 copies of every walk entry, shifted to
+    // the other lane quarters, let one accumulator cover 2 or 4 column tiles (see launch_spmm_tc)
+    L.stack = 1;
+    if (L.nst == 1 && g.bm < kTileM) L.stack = g.rows <= 32 ? 4 : (g.rows <= 64 ? 2 : 1);
     L.a_bytes = (uint32_t)(kTileM * g.bk * 2) / (sparse ? 2 : 1);
     L.entry_bytes = L.a_bytes + (sparse ? kMetaBytes : 0);
     L.walk_col_off = 0;
@@ -816,7 +838,7 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
     // the index of that side's own walk entry (or -1)
     L.npairs = (L.nst + 1) / 2;
     L.pwcap = (int)(2 * (int64_t)L.wcap < g.nblk ? 2 * L.wcap : g.nblk);
-    L.pair_col_off = L.image_off + align_up((size_t)L.nst * L.wcap * L.entry_bytes + 16);
+    L.pair_col_off = L.image_off + align_up((size_t)L.stack * L.nst * L.wcap * L.entry_bytes + 16);
     L.pair_len_off = L.pair_col_off + align_up((size_t)L.npairs * L.pwcap * sizeof(int32_t) + 4);
     L.pair_src_off = L.pair_len_off + align_up((size_t)L.npairs * sizeof(int32_t) + 4);
     L.total_bytes = L.pair_src_off + align_up((size_t)L.npairs * L.pwcap * 2 * sizeof(int32_t) + 4);
@@ -835,7 +857,7 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
                                                   reinterpret_cast<int32_t *>(d_exec + L.pair_len_off),
                                                   reinterpret_cast<int32_t *>(d_exec + L.pair_src_off));
     if (tiles_done) return cudaGetLastError();       // the encode kernel already wrote the weight tiles
-    const int grid = L.nst * L.wcap;
+    const int grid = L.stack * L.nst * L.wcap;
     const size_t smem_img = (size_t)L.entry_bytes + (size_t)g.vals_per_block() * 2 + (size_t)(g.vals_per_block() * g.idx_bits / 32) * 4 + 16;
     if (smem_img > 48 * 1024) {      // large blocks with many kept values need the opt-in shared memory size
         cudaError_t e = sparse ? cudaFuncSetAttribute(build_image_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_img)
@@ -843,10 +865,10 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
         if (e != cudaSuccess) return e;
     }
     if (sparse)
-        build_image_kernel<true><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
+        build_image_kernel<true><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.nst, L.wcap, L.stack, walk_col,
                                                                     walk_len, L.a_bytes, L.entry_bytes, image);
     else
-        build_image_kernel<false><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.wcap, walk_col,
+        build_image_kernel<false><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.nst, L.wcap, L.stack, walk_col,
                                                                      walk_len, L.a_bytes, L.entry_bytes, image);
     return cudaGetLastError();
 }
@@ -875,14 +897,19 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     int nt = (nt_override >= 1 && nt_override <= 4) ? nt_override : 4;
     const int64_t boxes = (ncols + kBoxN - 1) / kBoxN;
     if (boxes < nt) nt = (int)boxes;
+    // thin layers: a tile covers `stack` column tiles (one per group of accumulator lanes); not for the gather
+    // (only where it pays: walks that stay short when repeated per group, and enough columns to keep every SM busy)
+    int stack = conv ? 1 : L.stack;
+    if (stack > 1 && (L.wcap * stack > 8 || (ncols + stack * nt * kBoxN - 1) / (stack * nt * kBoxN) < sm_count)) stack = 1;
+    const int wlen = L.wcap * stack;                       // blocks per tile
     // small layers are latency-bound: narrower tiles (down to 2 boxes) until at least half of the SMs have one
     if (nt_override <= 0)
-        while (nt > 2 && (int64_t)L.nst * ((ncols + nt * kBoxN - 1) / (nt * kBoxN)) < sm_count / 2) --nt;
+        while (nt > 2 && (int64_t)L.nst * ((ncols + stack * nt * kBoxN - 1) / (stack * nt * kBoxN)) < sm_count / 2) --nt;
     // Short walks: the epilogue and the accumulator hand-over are the longest chain.  One warp per 64-column
     // box and lane quarter; under the sparse image three boxes, so that two accumulators fit beside the
     // metadata columns and the next tile's MMAs do not wait for the drain.
-    const bool short_walk = L.wcap <= 8 && nt_override <= 0;
-    if (short_walk && L.wcap <= 2 && sparse && nt == 4 && !conv) nt = 3;
+    const bool short_walk = wlen <= 8 && nt_override <= 0;
+    if (short_walk && wlen <= 2 && sparse && nt == 4 && !conv) nt = 3;
     TcParams p = {};
     if (conv) {
         // Pixel box of a column tile: tw * th * tb = 256 (or 128) output pixels, tw a power of two that divides
@@ -914,8 +941,9 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.walk_len = reinterpret_cast<const int32_t *>(d_exec + L.walk_len_off);
     p.status = d_status;
     p.bias = epilogue.bias; p.relu = epilogue.relu;
+    p.stack = stack;
     p.nst = L.nst; p.wcap = L.wcap; p.bk = g.bk; p.rows = g.rows; p.ncols = ncols; p.y = d_y; p.ldy = ldy;
-    p.n_col_tiles = (int)((ncols + nt * kBoxN - 1) / (nt * kBoxN));
+    p.n_col_tiles = (int)((ncols + stack * nt * kBoxN - 1) / (stack * nt * kBoxN));
     if (conv) p.n_col_tiles = p.cv_tiles_x * p.cv_tiles_y * ((conv->batch + p.cv_tb - 1) / p.cv_tb);
     const int64_t tiles = (int64_t)p.n_col_tiles * L.nst;
     if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
@@ -930,7 +958,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     const uint32_t epi = short_walk && nt >= 3 ? 4u * (uint32_t)nt : 8u;
     const uint32_t fixed = epi * kWideStageBytes + 256;
     uint32_t stages = (avail - fixed) / p.stage_bytes;
-    const uint32_t max_stages = p.stage_bytes <= 24 * 1024 ? (L.wcap <= 8 ? 6u : 7u) : (L.wcap <= 8 ? 4u : 8u);
+    const uint32_t max_stages = p.stage_bytes <= 24 * 1024 ? (wlen <= 8 ? 6u : 7u) : (wlen <= 8 ? 4u : 8u);
     if (stages > max_stages) stages = max_stages;
     if (stages < 2) return cudaErrorInvalidValue;
     p.num_stages = stages;
@@ -947,7 +975,7 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
                         (p.walk_cache ? cache_bytes : 0);
 
     CUtensorMap mx, my, ma;
-    p.a_map = make_map_image(&ma, p.image, (uint64_t)L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
+    p.a_map = make_map_image(&ma, p.image, (uint64_t)L.stack * L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
     if (!p.a_map) ma = CUtensorMap{};
     const bool f32 = y_dtype != 0;
     p.stg_swz_mask = 7;

@@ -36,7 +36,8 @@ CASES = [
     (200, 576, 333, 1, 4, 64, 64, 0.25),      # ragged rows and columns
     (96, 144, 1000, 2, 8, 32, 32, 0.5),       # short walks: 12 or 16 epilogue warps
     (300, 640, 520, 3, 4, 128, 64, 0.75),     # dense-tile image
-    (32, 32, 2048, 2, 8, 32, 32, 1.0),        # one lane quarter, three-box tiles
+    (32, 32, 2048, 2, 8, 32, 32, 1.0),        # thin layer: four column tiles per accumulator
+    (64, 384, 1300, 2, 8, 32, 32, 0.5),       # thin layer: two column tiles per accumulator, ragged columns
 ]
 
 

@@ -48,6 +48,12 @@ CASES = [
     (384, 768, 576, 2, 4, 128, 64, 0.5),     # 3 CTA tiles (odd: one pair has a ghost side), 2.25 column tiles
     (512, 512, 320, 1, 4, 64, 64, 0.25),
     (256, 256, 128, 2, 8, 32, 32, 0.5),
+    # thin layers (one CTA tile of at most 32 / 64 rows): a tile covers 4 / 2 column tiles, one per lane group
+    (16, 32, 5000, 2, 8, 32, 32, 1.0),
+    (24, 96, 3000, 2, 8, 32, 32, 0.67),
+    (32, 192, 4100, 2, 4, 32, 64, 0.5),
+    (64, 192, 2500, 2, 8, 32, 32, 0.5),      # two row tiles of 32 in the 64-row window
+    (48, 256, 1111, 3, 4, 64, 64, 0.5),      # dense-tile image, 48 of 64 rows
 ]
 
 
