@@ -57,7 +57,12 @@ def pick_layer(name: str) -> wl.Layer:
 # --------------------------------------------------------------------- clock sampling
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons while the timed region runs.
+
+    NVML is read in-process (a sample costs microseconds, so even a timed region of a few milliseconds is
+    covered): by a thread every 2 ms and by `sample()` calls from the timing loop itself.  Where NVML cannot
+    be loaded, `nvidia-smi -lms` is read instead.  Reading only: no setting of the GPU is touched.
+    """
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -66,8 +71,47 @@ class ClockSampler:
         self.uuid = uuid
         self.proc = None
         self.lines = []
+        self.nv = None
+        self.handle = None
+        self.sm, self.smax, self.reasons = [], [], set()
+        self._stop = threading.Event()
+        self._lock = threading.Lock()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if isinstance(uuid, str) else uuid)
+            self.nv = pynvml
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        nv = self.nv
+        if nv is None:
+            return
+        try:
+            mhz = float(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+            bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+        except Exception:
+            return
+        with self._lock:
+            self.sm.append(mhz)
+            self.smax.append(self.max_mhz)
+            for nm, bit in (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40),
+                            ("sw_thermal_slowdown", 0x20), ("sw_power_cap", 0x4)):
+                if bits & bit:
+                    self.reasons.add(nm)
+
+    def _poll(self):
+        while not self._stop.is_set():
+            self.sample()
+            time.sleep(0.002)
 
     def start(self):
+        if self.nv is not None:
+            self.t = threading.Thread(target=self._poll, daemon=True)
+            self.t.start()
+            return
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50"],
@@ -82,6 +126,12 @@ class ClockSampler:
             self.lines.append(line.strip())
 
     def stop(self):
+        if self.nv is not None:
+            self._stop.set()
+            self.t.join(timeout=1)
+            return {"sm_mhz": float(np.median(self.sm)) if self.sm else None,
+                    "sm_max_mhz": float(max(self.smax)) if self.smax else None,
+                    "samples": len(self.sm), "reasons": sorted(self.reasons), "source": "nvml"}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.06)
@@ -105,7 +155,7 @@ class ClockSampler:
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None,
                 "sm_max_mhz": float(max(smax)) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi"}
 
 
 # ------------------------------------------------------------------------ CPU oracle
@@ -456,6 +506,8 @@ def run_ours(args, layer, rank, world):
         ev[i][2].record(stream)
         L.spmm(d_x, y=d_y)
         ev[i][3].record(stream)
+        sampler.sample()                           # the stream is busy with the steps queued so far
+    sampler.sample()
     barrier()
     clocks = sampler.stop()
     t_mask = np.array([e[0].elapsed_time(e[1]) for e in ev])
