@@ -60,7 +60,8 @@ class ClockSampler:
     """Samples SM clock and throttle reasons while the timed region runs.
 
     NVML is read in-process (a sample costs microseconds, so even a timed region of a few milliseconds is
-    covered): by a thread every 2 ms and by `sample()` calls from the timing loop itself.  Where NVML cannot
+    covered): by a thread every 0.5 ms and by one `sample()` call after the last step has been queued (none
+    inside the loop: a slow host call there would let the GPU run dry between the launches of a step).  Where NVML cannot
     be loaded, `nvidia-smi -lms` is read instead.  Reading only: no setting of the GPU is touched.
     """
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -105,7 +106,7 @@ class ClockSampler:
     def _poll(self):
         while not self._stop.is_set():
             self.sample()
-            time.sleep(0.002)
+            time.sleep(0.0005)
 
     def start(self):
         if self.nv is not None:
@@ -506,8 +507,7 @@ def run_ours(args, layer, rank, world):
         ev[i][2].record(stream)
         L.spmm(d_x, y=d_y)
         ev[i][3].record(stream)
-        sampler.sample()                           # the stream is busy with the steps queued so far
-    sampler.sample()
+    sampler.sample()                               # the stream is still busy with the steps queued above
     barrier()
     clocks = sampler.stop()
     t_mask = np.array([e[0].elapsed_time(e[1]) for e in ev])
