@@ -60,8 +60,8 @@ class ClockSampler:
     """Samples SM clock and throttle reasons while the timed region runs.
 
     NVML is read in-process (a sample costs microseconds, so even a timed region of a few milliseconds is
-    covered): by a thread every 0.5 ms and by one `sample()` call after the last step has been queued (none
-    inside the loop: a slow host call there would let the GPU run dry between the launches of a step).  Where NVML cannot
+    covered): by a thread every 0.5 ms and by `sample()` calls placed between steps (after a step has been queued in
+    full, never between the launches of a step: a slow host call there would let the GPU run dry mid-step).  Where NVML cannot
     be loaded, `nvidia-smi -lms` is read instead.  Reading only: no setting of the GPU is touched.
     """
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -507,6 +507,9 @@ def run_ours(args, layer, rank, world):
         ev[i][2].record(stream)
         L.spmm(d_x, y=d_y)
         ev[i][3].record(stream)
+        if i % 4 == 3:
+            sampler.sample()                       # between steps: step i is queued in full, so no launch of a
+                                                   # step waits for this host call
     sampler.sample()                               # the stream is still busy with the steps queued above
     barrier()
     clocks = sampler.stop()
