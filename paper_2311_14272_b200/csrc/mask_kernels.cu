@@ -35,9 +35,10 @@ __device__ __forceinline__ void load8_raw(const float *__restrict__ s, int64_t l
     key[0] = a.x; key[1] = a.y; key[2] = a.z; key[3] = a.w;
     key[4] = b.x; key[5] = b.y; key[6] = b.z; key[7] = b.w;
 }
+// |s| with NaN -> 0 and Inf -> FLT_MAX in two instructions: max(|s|, 0) drops a NaN (the maximum of a NaN and a
+// number is the number), min(., FLT_MAX) caps infinity; -0 becomes +0, denormals pass unchanged.
 __device__ __forceinline__ uint32_t canonical_bits(uint32_t u) {
-    u &= 0x7FFFFFFFu;
-    return u > 0x7F800000u ? 0u : min(u, 0x7F7FFFFFu);
+    return __float_as_uint(fminf(fmaxf(fabsf(__uint_as_float(u)), 0.f), 3.402823466e+38f));
 }
 
 // Eight consecutive saliency values of one row, zero beyond the matrix.
