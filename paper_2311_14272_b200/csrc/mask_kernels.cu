@@ -166,8 +166,8 @@ constexpr int kM1RowsPerWarp = kM1Rows / (kM1Threads / 32);
 
 // K-M1.  One CTA covers 32 rows x 256 k-elements.  Warp w takes rows 4w..4w+3 (all loads issued
 // first); lane l owns the 8 elements at k = chunk*256 + 8*l of each row, so a lane stays inside one
-// block column and keeps its partial block score in a register.  Four lanes assemble one 32-bit
-// mask word and one partial score (a word never straddles a block: block_k is a multiple of 32).
+// block column and keeps its partial block score in a register.  A lane stores its eight mask bits as
+// one byte; four lanes add up one partial score (a word never straddles a block: block_k is a multiple of 32).
 template <int M>
 __global__ void __launch_bounds__(kM1Threads)
 group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_ok,
@@ -225,10 +225,9 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
             for (int j = 0; j < 8; ++j)
                 if ((counted >> j) & 1u) acc += fixed_point_score(key[i][j], e_max);
         }
-        uint32_t word = bits << (8 * (lane & 3));
-        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-        if ((lane & 3) == 0 && in_kp) nm_bits[row * g.wpr + (k0 >> 5)] = word;
+        // the lane's eight bits are byte (k0 / 8) mod 4 of their little-endian mask word: a warp stores 32
+        // consecutive bytes of the row
+        if (in_kp) reinterpret_cast<uint8_t *>(nm_bits + row * g.wpr)[k0 >> 3] = (uint8_t)bits;
     }
     acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
     acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
