@@ -6,6 +6,7 @@
 #include <vector>
 
 #include "crisp_internal.h"
+#include "walks.cuh"
 
 using crisp::align_up;
 using crisp::Geometry;
@@ -181,13 +182,18 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     const bool fuse_tiles = h->exec_kind != CRISP_PATH_DIRECT && g.bm == 128;
     crisp::TcImageLayout L = {};
     if (h->exec_kind != CRISP_PATH_DIRECT) L = crisp::tc_image_layout(g, h->exec_kind == CRISP_PATH_SPARSE);
+    // the walk lists of the tensor-core kernel depend on the mask only: CTAs of the encode kernel build them
+    const bool tc = h->exec_kind != CRISP_PATH_DIRECT;
+    crisp::WalkArgs walks = {};
+    if (tc) walks = crisp::tc_walk_args(g, h->exec_kind == CRISP_PATH_SPARSE, mask->d_blk_col, h->d_exec);
     if (e == cudaSuccess)
         e = crisp::launch_encode_canonical(d_w_bf16, ld_w, g, mask->d_blk_col, mask->d_nm_bits,
                                            h->d_blk_col, h->d_vals, h->d_idx, fuse_tiles ? h->exec_kind : 0,
-                                           fuse_tiles ? h->d_exec + L.image_off : nullptr, L.a_bytes, L.entry_bytes, st);
-    if (e == cudaSuccess && h->exec_kind != CRISP_PATH_DIRECT)
+                                           fuse_tiles ? h->d_exec + L.image_off : nullptr, L.a_bytes, L.entry_bytes,
+                                           tc ? &walks : nullptr, st);
+    if (e == cudaSuccess && tc)
         e = crisp::launch_build_image(g, h->exec_kind == CRISP_PATH_SPARSE, h->d_blk_col, h->d_vals, h->d_idx,
-                                      h->d_exec, fuse_tiles, st);
+                                      h->d_exec, fuse_tiles, /*walks_done=*/true, st);
     if (e != cudaSuccess) { delete h; return CRISP_CUDA_ERROR; }
     *out = h;
     return CRISP_OK;

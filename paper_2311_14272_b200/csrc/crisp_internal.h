@@ -59,6 +59,8 @@ struct crisp_handle_s {
 
 namespace crisp {
 
+struct WalkArgs;
+
 // mask_kernels.cu
 cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, int32_t *d_blk_col,
                               uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes,
@@ -70,7 +72,7 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
                                     const int32_t *d_mask_blk_col, const uint32_t *d_nm_bits,
                                     int32_t *d_blk_col, uint16_t *d_vals, uint32_t *d_idx,
                                     int tile_kind, uint8_t *d_image, uint32_t a_bytes, uint32_t entry_bytes,
-                                    cudaStream_t st);
+                                    const struct WalkArgs *walks, cudaStream_t st);
 cudaError_t launch_decode(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                           const uint32_t *d_idx, uint16_t *d_w, int64_t ld, cudaStream_t st);
 
@@ -89,8 +91,12 @@ struct TcImageLayout {
 };
 bool tc_pattern_is_sparse(const Geometry &g);
 TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
+// walk lists of the tensor-core kernel (walks.cuh): built by CTAs of the encode kernel (walks != nullptr in
+// launch_encode_canonical, then walks_done below) or by a kernel of their own
+struct WalkArgs tc_walk_args(const Geometry &g, bool sparse, const int32_t *d_mask_blk_col, uint8_t *d_exec);
 cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
-                               const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, cudaStream_t st);
+                               const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, bool walks_done,
+                               cudaStream_t st);
 bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols);
 // Convolution geometry for the implicit-GEMM mode (stride 1): NHWC activation, ho x wo output pixels.
 struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo; };

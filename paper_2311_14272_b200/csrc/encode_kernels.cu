@@ -1,6 +1,7 @@
 // Canonical compressed format of Sec. III-A: kept-block column list (Blocked-ELLPACK) plus,
 // per kept value, its bf16 payload and a log2(M)-bit zero-based offset inside its M-vector.
 #include "crisp_internal.h"
+#include "walks.cuh"
 
 namespace crisp {
 
@@ -44,9 +45,16 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
                     const int32_t *__restrict__ mask_blk_col, const uint32_t *__restrict__ nm_bits,
                     int32_t *__restrict__ blk_col, uint16_t *__restrict__ vals,
                     uint32_t *__restrict__ idx, uint8_t *__restrict__ image, uint32_t a_bytes,
-                    uint32_t entry_bytes) {
+                    uint32_t entry_bytes, WalkArgs walks) {
     extern __shared__ uint32_t s_buf[];
-    const int blk = blockIdx.x;                       // rt * kkeep + slot
+    // The first walks.npairs CTAs build the walk lists of the tensor-core kernel instead of encoding a block:
+    // that needs only the mask's block list, so it overlaps the encoding instead of following it.
+    if ((int)blockIdx.x < walks.npairs) {
+        __shared__ WalkShared s_walks;
+        build_walks_body(g, walks, blockIdx.x, s_walks);
+        return;
+    }
+    const int blk = (int)blockIdx.x - walks.npairs;   // rt * kkeep + slot
     const int rt = blk / g.kkeep;
     const int jb = mask_blk_col[blk];
     const int groups = g.bk / M;
@@ -174,9 +182,11 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
                                     const int32_t *d_mask_blk_col, const uint32_t *d_nm_bits,
                                     int32_t *d_blk_col, uint16_t *d_vals, uint32_t *d_idx,
                                     int tile_kind, uint8_t *d_image, uint32_t a_bytes, uint32_t entry_bytes,
-                                    cudaStream_t st) {
+                                    const WalkArgs *walks, cudaStream_t st) {
     const int nblocks = g.nrt * g.kkeep;
     if (nblocks == 0) return cudaSuccess;
+    WalkArgs wa = {};
+    if (walks) wa = *walks;
     const size_t vpb = (size_t)g.vals_per_block();
     size_t smem = (vpb * g.idx_bits / 32) * sizeof(uint32_t) + (vpb + 7) / 8 * 16 + 16;
     if (tile_kind != 0) smem += entry_bytes;
@@ -190,8 +200,8 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
             if (e != cudaSuccess) return e;                                                                  \
         }                                                                                                    \
-        kern<<<nblocks, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits, d_blk_col, d_vals,   \
-                                         d_idx, d_image, a_bytes, entry_bytes);                              \
+        kern<<<nblocks + wa.npairs, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits, d_blk_col, \
+                                                     d_vals, d_idx, d_image, a_bytes, entry_bytes, wa);      \
     } while (0)
     if (g.m == 4) {
         if (tile_kind == CRISP_PATH_SPARSE) CRISP_ENCODE_LAUNCH(4, CRISP_PATH_SPARSE);

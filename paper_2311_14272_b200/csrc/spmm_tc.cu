@@ -17,6 +17,7 @@
 
 #include "crisp_internal.h"
 #include "tc_common.cuh"
+#include "walks.cuh"
 
 namespace crisp {
 
@@ -533,62 +534,11 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
 // --------------------------------------------------------------------- execution image kernels
 
-// Walk lists.  One CTA per pair of adjacent 128-row CTA tiles:
-//   walk of a CTA tile  = ascending union of the kept block columns of its r = 128 / bm row tiles;
-//   walk of the pair    = ascending union of its two CTA tiles' walks, with each side's entry index
-//                         (or -1) for the CTA-pair kernel.
-// Kept columns are marked in shared bitmaps and compacted with a prefix over the bitmap words.
+// Walk lists as a kernel of their own (the body, and what it builds, are described in walks.cuh).
 __global__ void __launch_bounds__(256)
-build_walks_kernel(Geometry g, const int32_t *__restrict__ blk_col, int r, int nst, int wcap, int pwcap,
-                   int32_t *__restrict__ walk_col, int32_t *__restrict__ walk_len,
-                   int32_t *__restrict__ pair_col, int32_t *__restrict__ pair_len, int32_t *__restrict__ pair_src) {
-    __shared__ uint32_t s_bits[2][128];              // nblk <= 4096
-    __shared__ int s_prefix[3][129];
-    const int p = blockIdx.x;
-    const int words = (g.nblk + 31) / 32;
-    for (int i = threadIdx.x; i < 2 * 128; i += blockDim.x) s_bits[i >> 7][i & 127] = 0u;
-    __syncthreads();
-    for (int side = 0; side < 2; ++side) {
-        const int st = 2 * p + side;
-        if (st >= nst) continue;
-        const int first_rt = st * r;
-        const int n_rt = min(r, g.nrt - first_rt);
-        for (int i = threadIdx.x; i < n_rt * g.kkeep; i += blockDim.x) {
-            const int jb = blk_col[(int64_t)first_rt * g.kkeep + i];
-            atomicOr(&s_bits[side][jb >> 5], 1u << (jb & 31));
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < 3) {                           // prefix of side 0, side 1 and of their union
-        const int which = threadIdx.x;
-        int run = 0;
-        for (int i = 0; i < words; ++i) {
-            s_prefix[which][i] = run;
-            const uint32_t b = which == 2 ? (s_bits[0][i] | s_bits[1][i]) : s_bits[which][i];
-            run += __popc(b);
-        }
-        if (which == 2) pair_len[p] = run;
-        else if (2 * p + which < nst) walk_len[2 * p + which] = run;
-    }
-    __syncthreads();
-    for (int jb = threadIdx.x; jb < g.nblk; jb += blockDim.x) {
-        const int w = jb >> 5;
-        const uint32_t below = (1u << (jb & 31)) - 1u;
-        int pos[2] = {-1, -1};
-        for (int side = 0; side < 2; ++side) {
-            const uint32_t b = s_bits[side][w];
-            if ((b >> (jb & 31)) & 1u) {
-                pos[side] = s_prefix[side][w] + __popc(b & below);
-                walk_col[(int64_t)(2 * p + side) * wcap + pos[side]] = jb;
-            }
-        }
-        if (pos[0] >= 0 || pos[1] >= 0) {
-            const int o = s_prefix[2][w] + __popc((s_bits[0][w] | s_bits[1][w]) & below);
-            pair_col[(int64_t)p * pwcap + o] = jb;
-            pair_src[((int64_t)p * pwcap + o) * 2 + 0] = pos[0];
-            pair_src[((int64_t)p * pwcap + o) * 2 + 1] = pos[1];
-        }
-    }
+build_walks_kernel(Geometry g, WalkArgs a) {
+    __shared__ WalkShared sh;
+    build_walks_body(g, a, blockIdx.x, sh);
 }
 
 // One CTA per walk entry: assemble the entry's weight tile (and 2:4 metadata) in shared memory from
@@ -845,17 +795,29 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
     return L;
 }
 
+WalkArgs tc_walk_args(const Geometry &g, bool sparse, const int32_t *d_blk_col, uint8_t *d_exec) {
+    const TcImageLayout L = tc_image_layout(g, sparse);
+    WalkArgs a;
+    a.blk_col = d_blk_col;
+    a.r = L.r; a.nst = L.nst; a.wcap = L.wcap; a.pwcap = L.pwcap;
+    a.npairs = g.nrt * g.kkeep == 0 ? 0 : L.npairs;
+    a.walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
+    a.walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
+    a.pair_col = reinterpret_cast<int32_t *>(d_exec + L.pair_col_off);
+    a.pair_len = reinterpret_cast<int32_t *>(d_exec + L.pair_len_off);
+    a.pair_src = reinterpret_cast<int32_t *>(d_exec + L.pair_src_off);
+    return a;
+}
+
 cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
-                               const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, cudaStream_t st) {
+                               const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, bool walks_done,
+                               cudaStream_t st) {
     const TcImageLayout L = tc_image_layout(g, sparse);
     if (g.nrt * g.kkeep == 0) return cudaSuccess;
     int32_t *walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
     int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
     uint8_t *image = d_exec + L.image_off;
-    build_walks_kernel<<<L.npairs, 256, 0, st>>>(g, d_blk_col, L.r, L.nst, L.wcap, L.pwcap, walk_col, walk_len,
-                                                  reinterpret_cast<int32_t *>(d_exec + L.pair_col_off),
-                                                  reinterpret_cast<int32_t *>(d_exec + L.pair_len_off),
-                                                  reinterpret_cast<int32_t *>(d_exec + L.pair_src_off));
+    if (!walks_done) build_walks_kernel<<<L.npairs, 256, 0, st>>>(g, tc_walk_args(g, sparse, d_blk_col, d_exec));
     if (tiles_done) return cudaGetLastError();       // the encode kernel already wrote the weight tiles
     const int grid = L.stack * L.nst * L.wcap;
     const size_t smem_img = (size_t)L.entry_bytes + (size_t)g.vals_per_block() * 2 + (size_t)(g.vals_per_block() * g.idx_bits / 32) * 4 + 16;
