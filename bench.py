@@ -640,7 +640,7 @@ def run_ours(args, layer, rank, world):
 
     # mask: max_key, group_select, block_select; encode: encode_block (+ tiles for 128-row blocks), walk lists,
     # and a separate image kernel for narrower blocks; spmm: one persistent kernel
-    kernels_per_step = {"mask": 3, "encode": 2 if layer.block_rows == 128 else 3, "spmm": 1}
+    kernels_per_step = {"mask": 3, "encode": 1 if layer.block_rows == 128 else 2, "spmm": 1}
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
