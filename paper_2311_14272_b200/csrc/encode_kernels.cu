@@ -40,7 +40,7 @@ __device__ __forceinline__ void load_group(const uint16_t *__restrict__ w, int64
 // 0 nothing, CRISP_PATH_DENSE the zero-expanded tile, CRISP_PATH_SPARSE the 2:4 compressed tile with
 // its metadata (layouts: see the execution-image kernels of the tensor-core SpMM).
 template <int M, int TILE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 8)
 encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool vec_ok,
                     const int32_t *__restrict__ mask_blk_col, const uint32_t *__restrict__ nm_bits,
                     int32_t *__restrict__ blk_col, uint16_t *__restrict__ vals,
