@@ -96,6 +96,21 @@ typedef struct {
 #define CRISP_PATH_DENSE  1   /* tcgen05 dense MMA over zero-expanded kept blocks            */
 #define CRISP_PATH_SPARSE 2   /* tcgen05 sparse (2:4) MMA over compressed kept blocks        */
 
+/* What the last crisp_spmm / crisp_spmm_conv on a handle really launched (crisp_last_launch).
+ * `path` is the kernel family that ran, which differs from crisp_bytes_t.path when the operands
+ * of that call could not be addressed by the tensor-core kernel (Sec. III-E is the same three
+ * steps on every path). */
+typedef struct {
+    int32_t path;             /* CRISP_PATH_* of the kernel that was launched, -1 before any    */
+    int32_t tile_cols;        /* columns of X / Y per CTA tile (0 on the direct path)           */
+    int32_t accumulators;     /* tensor-memory accumulators per CTA                              */
+    int32_t stack;            /* column tiles stacked in one accumulator (thin layers), else 1   */
+    int32_t epilogue_warps;
+    int32_t stages;           /* depth of the shared-memory ring                                 */
+    int32_t ctas;             /* grid size                                                       */
+    int32_t conv;             /* 1 if the activations were gathered from an NHWC tensor          */
+} crisp_launch_info_t;
+
 /* kkeep = floor(keep_ratio * nblk + 0.5), clamped to [0, nblk], evaluated in double on the
  * host.  This is the "select by the current sparsity target" step of Algorithm 1 with the
  * per-layer ratio given by the caller.  Error: INVALID_ARG / BAD_SHAPE / UNSUPPORTED. */
@@ -135,15 +150,19 @@ CRISP_API crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s,
  *
  * The scratch lives in a fixed array of CRISP_STATIC_SCRATCH_BYTES inside the library image;
  * every GPU that loads the library holds it until the process exits.  The call allocates and
- * frees nothing, on host-visible CUDA APIs or otherwise.  Inputs and outputs are still the
- * caller's: d_saliency, d_mask_buf (crisp_mask_sizes gives its size) and the returned mask.
+ * frees no device memory and calls no allocating CUDA routine; the only allocation is the small
+ * host object behind the returned crisp_mask_t (a few dozen bytes from the C++ heap, freed by
+ * crisp_mask_destroy).  Inputs and outputs are still the caller's: d_saliency, d_mask_buf
+ * (crisp_mask_sizes gives its size) and the returned mask.
  *
  * Limits and rules
  *   - The layer's workspace (256 bytes + 8 bytes per coarse block, i.e. per (row tile,
  *     k-block) pair) must fit: at most 32736 coarse blocks.  Larger layers are refused with
  *     CRISP_BUFFER_TOO_SMALL before anything is launched; use crisp_build_mask for them.
- *   - The first call on each device looks up the array's device address (with that device
- *     current).  Make that first call during set-up, before any stream capture begins.
+ *   - Every call looks up the array's device address with the current device current; the first
+ *     call on a device also makes the runtime load the library's module there.  Make that first
+ *     call during set-up, before any stream capture begins.  The address is never kept across
+ *     calls, so cudaDeviceReset or a second context on the device cannot leave a stale one.
  *   - All calls on a device share the one array, and it keeps what the last call wrote.  Each
  *     call clears it on `stream` before use, so calls issued one after another on the same
  *     stream are safe; calls that may run concurrently on the GPU (different streams or host
@@ -199,7 +218,9 @@ CRISP_API crisp_status_t crisp_saliency_finish(const float *d_acc, int64_t ld_ac
  *
  * layers (host array) is read before the call returns.  d_workspace: crisp_global_rank_sizes
  * bytes, 256-byte aligned, scratch.  d_kkeep: device, int32 [n_layers], written on `stream`.
- * nblk <= 4096 per layer (CRISP_UNSUPPORTED beyond).  Nothing is allocated.
+ * nblk <= 4096 per layer (CRISP_UNSUPPORTED beyond).  No device memory is allocated; the layer table is
+ * staged through a small temporary host array, so the call is refused (CRISP_UNSUPPORTED) while
+ * `stream` is being captured into a graph.
  */
 typedef struct {
     const unsigned long long *d_scores;  /* device, [nrt, nblk] block scores                      */
@@ -317,6 +338,24 @@ CRISP_API crisp_status_t crisp_set_epilogue(crisp_handle_t handle, const float *
 /* Restrict crisp_spmm of this handle to one kernel family (CRISP_PATH_*), or -1 for the
  * default choice.  UNSUPPORTED if the handle's execution image cannot serve that path. */
 CRISP_API crisp_status_t crisp_set_path(crisp_handle_t h, int32_t path);
+
+/* Kernel family and tile configuration of the last product launched through this handle. */
+CRISP_API crisp_status_t crisp_last_launch(crisp_handle_t h, crisp_launch_info_t *out);
+
+/* Tuning and failure-detection controls of the tensor-core kernels of this handle (all optional).
+ *   tile_boxes        64-column boxes per CTA tile, 1..4; 0 = chosen by the library
+ *   wait_limit_cycles every wait inside the kernel (on a pipeline stage, on an accumulator) gives
+ *                     up after this many SM cycles, the kernel then lets its copies land, frees its
+ *                     tensor memory, returns, and the device status reads CRISP_TIMEOUT; 0 = the
+ *                     default of about two seconds
+ *   skip_fill         test hook, -1 = off: every CTA leaves out the loads of its skip_fill-th
+ *                     pipeline fill, so that the wait for them expires (use with a short limit)
+ * The paper has no counterpart; Sec. III-E's pipeline has no failure model. */
+CRISP_API crisp_status_t crisp_set_tuning(crisp_handle_t h, int32_t tile_boxes, uint64_t wait_limit_cycles,
+                                          int32_t skip_fill);
+
+/* Clear the device status word of the handle on `stream` (after a reported CRISP_TIMEOUT). */
+CRISP_API crisp_status_t crisp_reset_status(crisp_handle_t h, void *stream);
 
 /* Read the device status word of the handle (0 = no kernel reported a problem; otherwise a
  * crisp_status_t, e.g. CRISP_TIMEOUT when a bounded wait expired).  Synchronises `stream`. */

@@ -22,7 +22,7 @@
  *     product; the oracle is that definition: decode, then an fp64 triple loop;
  *     for a convolution layer, the definition of the convolution (no lowering).
  *
- * Readings where the paper is silent (mirrored in the design notes):
+ * Readings where the paper is silent:
  *   rows of W are output channels and groups/blocks run along the reduction
  *   dimension; ties go to the lower index; saliency enters as |s| with NaN -> 0
  *   and Inf -> FLT_MAX; the block score is an exact fixed-point integer sum so

@@ -34,6 +34,14 @@ class ConvDesc(C.Structure):
                 ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad", C.c_int32)]
 
 
+class LaunchInfo(C.Structure):
+    _fields_ = [("path", C.c_int32), ("tile_cols", C.c_int32), ("accumulators", C.c_int32), ("stack", C.c_int32),
+                ("epilogue_warps", C.c_int32), ("stages", C.c_int32), ("ctas", C.c_int32), ("conv", C.c_int32)]
+
+    def as_dict(self):
+        return {f: int(getattr(self, f)) for f, _ in self._fields_}
+
+
 class BytesModel(C.Structure):
     _fields_ = [("nnz", C.c_int64), ("vals_bytes", C.c_int64), ("idx_bytes", C.c_int64),
                 ("blk_col_bytes", C.c_int64), ("x_bytes", C.c_int64), ("y_bytes", C.c_int64),
@@ -85,6 +93,9 @@ def load(path: Optional[str] = None):
         "crisp_set_path": [vp, i32],
         "crisp_set_epilogue": [vp, vp, i32],
         "crisp_device_status": [vp, vp, P(i32)],
+        "crisp_last_launch": [vp, P(LaunchInfo)],
+        "crisp_set_tuning": [vp, i32, C.c_uint64, i32],
+        "crisp_reset_status": [vp, vp],
         "crisp_bytes_model": [vp, i64, i32, P(BytesModel)],
         "crisp_mask_scores": [P(LayerDesc), vp, P(vp), P(vp)],
         "crisp_global_rank_sizes": [i32, P(RankLayer), P(sz)],
@@ -275,6 +286,21 @@ def crisp_device_status(handle: int, stream=None) -> int:
     return s.value
 
 
+def crisp_last_launch(handle: int) -> dict:
+    """Kernel family (`path`) and tile configuration of the last product launched through the handle."""
+    info = LaunchInfo()
+    _check(load().crisp_last_launch(handle, C.byref(info)), "crisp_last_launch")
+    return info.as_dict()
+
+
+def crisp_set_tuning(handle: int, tile_boxes: int = 0, wait_limit_cycles: int = 0, skip_fill: int = -1):
+    _check(load().crisp_set_tuning(handle, tile_boxes, wait_limit_cycles, skip_fill), "crisp_set_tuning")
+
+
+def crisp_reset_status(handle: int, stream=None):
+    _check(load().crisp_reset_status(handle, _stream(stream)), "crisp_reset_status")
+
+
 def crisp_bytes_model(handle: int, ncols: int, y_dtype: int = 0) -> dict:
     b = BytesModel()
     _check(load().crisp_bytes_model(handle, ncols, y_dtype, C.byref(b)), "crisp_bytes_model")
@@ -407,6 +433,16 @@ class HybridLayer:
 
     def device_status(self, stream=None) -> int:
         return crisp_device_status(self.handle, stream)
+
+    def last_launch(self) -> dict:
+        return crisp_last_launch(self.handle)
+
+    def set_tuning(self, tile_boxes=0, wait_limit_cycles=0, skip_fill=-1):
+        crisp_set_tuning(self.handle, tile_boxes, wait_limit_cycles, skip_fill)
+        return self
+
+    def reset_status(self, stream=None):
+        crisp_reset_status(self.handle, stream)
 
     def bytes_model(self, ncols, y_dtype=0):
         return crisp_bytes_model(self.handle, ncols, y_dtype)

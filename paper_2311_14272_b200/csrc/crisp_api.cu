@@ -47,7 +47,8 @@ void fill_desc(const Geometry &g, double keep_ratio, crisp_layer_desc_t *d) {
 
 // Which execution image crisp_encode lays out.  Default: the 2:4 sparse-MMA image when every aligned
 // 4-group keeps at most two values (n <= 2), the zero-expanded dense-tile image otherwise.  The
-// environment variable CRISP_EXEC_IMAGE = dense | none overrides it (for measurements).
+// environment variable CRISP_EXEC_IMAGE = dense | none overrides it (for measurements).  Evaluated once
+// per mask, in crisp_build_mask, and carried by the mask from then on.
 int image_kind(const Geometry &g) {
     const char *e = std::getenv("CRISP_EXEC_IMAGE");
     if (e && !std::strcmp(e, "none")) return CRISP_PATH_DIRECT;
@@ -116,6 +117,7 @@ crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s, const cri
     mk->g = g;
     mk->d_blk_col = reinterpret_cast<int32_t *>(d_mask_buf);
     mk->d_nm_bits = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_mask_buf) + blk_col_bytes(g));
+    mk->image_kind = image_kind(g);
     cudaError_t e = crisp::launch_build_mask(d_saliency, ld_s, g, mk->d_blk_col, mk->d_nm_bits, d_workspace,
                                              crisp::mask_workspace_bytes(g), (cudaStream_t)stream);
     if (e != cudaSuccess) { delete mk; return CRISP_CUDA_ERROR; }
@@ -150,7 +152,7 @@ crisp_status_t crisp_encode_sizes(crisp_mask_t mask, size_t *canonical_bytes, si
     if (!mask) return CRISP_INVALID_ARG;
     const Geometry &g = mask->g;
     if (canonical_bytes) *canonical_bytes = blk_col_bytes(g) + vals_bytes(g) + idx_bytes(g);
-    if (exec_bytes) *exec_bytes = kAlign + exec_payload_bytes(g, image_kind(g));
+    if (exec_bytes) *exec_bytes = kAlign + exec_payload_bytes(g, mask->image_kind);
     return CRISP_OK;
 }
 
@@ -172,10 +174,16 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     h->d_idx = reinterpret_cast<uint32_t *>(p);
     h->d_status = reinterpret_cast<int32_t *>(d_exec_buf);
     h->d_exec = reinterpret_cast<uint8_t *>(d_exec_buf) + kAlign;
-    h->exec_kind = image_kind(g);
+    h->exec_kind = mask->image_kind;
     h->exec_payload_bytes = exec_payload_bytes(g, h->exec_kind);
     h->forced_path = -1;
     h->epilogue = crisp::Epilogue{nullptr, 0};
+    const char *nt_env = std::getenv("CRISP_TC_NT");          // 64-column boxes per CTA tile, tuning only; read once
+    h->nt_override = nt_env ? std::atoi(nt_env) : 0;
+    h->wait_limit_cycles = 0;
+    h->debug_skip_stage = -1;
+    h->plan = nullptr;
+    h->last = crisp_launch_info_t{-1, 0, 0, 1, 0, 0, 0, 0};
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
     // 128-row blocks: one kept block is one tensor-core tile, so the encode kernel writes it directly
@@ -258,17 +266,10 @@ crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ld
     if (path == CRISP_PATH_DIRECT) {
         e = crisp::launch_spmm_direct(h->g, h->d_blk_col, h->d_vals, h->d_idx, d_x_bf16, ldx, ncols,
                                       d_y, ldy, y_dtype, h->epilogue, (cudaStream_t)stream);
+        if (e == cudaSuccess) h->last = crisp_launch_info_t{CRISP_PATH_DIRECT, 0, 0, 1, 0, 0, 0, 0};
     } else {
-        const char *pair = std::getenv("CRISP_TC_PAIR");   // 1: CTA-pair kernel, 0: single-CTA kernel
-        const bool plain = h->epilogue.bias == nullptr && !h->epilogue.relu;      // the pair kernel has no layer epilogue
-        const bool use_pair = pair && std::atoi(pair) == 1 && plain && crisp::tc_pair_supported(h->g, ncols);
-        const char *nt = std::getenv("CRISP_TC_NT");     // column boxes per CTA tile, tuning only
-        if (use_pair)
-            e = crisp::launch_spmm_tc_pair(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx,
-                                           ncols, d_y, ldy, y_dtype, (cudaStream_t)stream);
-        else
-        e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_x_bf16, ldx, ncols,
-                                  d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, nullptr, h->epilogue, (cudaStream_t)stream);
+        e = crisp::launch_spmm_tc(h, path == CRISP_PATH_SPARSE, d_x_bf16, ldx, ncols, d_y, ldy, y_dtype, nullptr,
+                                  (cudaStream_t)stream);
     }
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }
@@ -293,11 +294,30 @@ crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, con
     if (!aligned(d_y, es)) return CRISP_INVALID_ARG;
     const int path = h->forced_path >= 0 ? h->forced_path : h->exec_kind;
     if (path == CRISP_PATH_DIRECT || h->g.kkeep == 0) return CRISP_UNSUPPORTED;
-    const char *nt = std::getenv("CRISP_TC_NT");
-    cudaError_t e = crisp::launch_spmm_tc(h->g, path == CRISP_PATH_SPARSE, h->d_exec, h->d_status, d_act_nhwc, 0, ncols,
-                                          d_y, ldy, y_dtype, nt ? std::atoi(nt) : 0, &cg, h->epilogue, (cudaStream_t)stream);
+    cudaError_t e = crisp::launch_spmm_tc(h, path == CRISP_PATH_SPARSE, d_act_nhwc, 0, ncols, d_y, ldy, y_dtype, &cg,
+                                          (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return CRISP_UNSUPPORTED;
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
+}
+
+crisp_status_t crisp_last_launch(crisp_handle_t h, crisp_launch_info_t *out) {
+    if (!h || !out) return CRISP_INVALID_ARG;
+    *out = h->last;
+    return CRISP_OK;
+}
+
+crisp_status_t crisp_set_tuning(crisp_handle_t h, int32_t tile_boxes, uint64_t wait_limit_cycles, int32_t skip_fill) {
+    if (!h || tile_boxes < 0 || tile_boxes > 4 || skip_fill < -1) return CRISP_INVALID_ARG;
+    h->nt_override = tile_boxes;
+    h->wait_limit_cycles = wait_limit_cycles;
+    h->debug_skip_stage = skip_fill;
+    return CRISP_OK;
+}
+
+crisp_status_t crisp_reset_status(crisp_handle_t h, void *stream) {
+    if (!h) return CRISP_INVALID_ARG;
+    return cudaMemsetAsync(h->d_status, 0, sizeof(int32_t), (cudaStream_t)stream) == cudaSuccess ? CRISP_OK
+                                                                                                 : CRISP_CUDA_ERROR;
 }
 
 crisp_status_t crisp_device_status(crisp_handle_t h, void *stream, int32_t *status_out) {
@@ -339,6 +359,9 @@ crisp_status_t crisp_bytes_model(crisp_handle_t h, int64_t ncols, int32_t y_dtyp
 }
 
 void crisp_mask_destroy(crisp_mask_t mask) { delete mask; }
-void crisp_destroy(crisp_handle_t h) { delete h; }
+void crisp_destroy(crisp_handle_t h) {
+    if (h) crisp::tc_plan_destroy(h->plan);
+    delete h;
+}
 
 }  // extern "C"

@@ -40,7 +40,16 @@ struct crisp_mask_s {
     crisp::Geometry g;
     int32_t *d_blk_col;     // [nrt, kkeep]
     uint32_t *d_nm_bits;    // [mp, wpr]
+    int image_kind;         // CRISP_PATH_* of the execution image crisp_encode will lay out: fixed when the
+                            // mask is built, so that crisp_encode_sizes and crisp_encode always agree
 };
+
+namespace crisp {
+// Launch plan of the tensor-core kernel for one set of operands (spmm_tc.cu); cached in the handle so that
+// repeated products on the same buffers skip the tensor-map encoding.
+struct TcPlan;
+void tc_plan_destroy(TcPlan *plan);
+}  // namespace crisp
 
 struct crisp_handle_s {
     crisp::Geometry g;
@@ -55,6 +64,11 @@ struct crisp_handle_s {
     int exec_kind;          // CRISP_PATH_* the image was laid out for (DIRECT = none)
     int forced_path;        // -1 = default
     crisp::Epilogue epilogue;
+    int nt_override;        // tuning: 64-column boxes per CTA tile (0 = chosen by the library)
+    unsigned long long wait_limit_cycles;   // bound of every in-kernel wait (0 = default)
+    int debug_skip_stage;   // test hook: the producer leaves out the loads of this pipeline fill (-1 = none)
+    crisp::TcPlan *plan;    // cached launch plan of the last tensor-core product (or nullptr)
+    crisp_launch_info_t last;               // what the last product on this handle launched
 };
 
 namespace crisp {
@@ -85,9 +99,6 @@ struct TcImageLayout {
     uint32_t a_bytes;       // weight tile bytes per walk entry
     uint32_t entry_bytes;   // weight tile + metadata
     size_t walk_col_off, walk_len_off, image_off, total_bytes;   // offsets inside the exec payload
-    int npairs;             // pairs of adjacent CTA tiles (CTA-pair kernel)
-    int pwcap;              // capacity of one pair's union walk list
-    size_t pair_col_off, pair_len_off, pair_src_off;
 };
 bool tc_pattern_is_sparse(const Geometry &g);
 TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
@@ -101,15 +112,9 @@ bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int 
 // Convolution geometry for the implicit-GEMM mode (stride 1): NHWC activation, ho x wo output pixels.
 struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo; };
 // conv == nullptr: d_x is the [k, ncols] matrix.  Otherwise d_x is the activation and ncols = batch*ho*wo.
-cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
-                           const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
-                           int nt_override, const ConvGeom *conv, const Epilogue &epi, cudaStream_t st);
-// spmm_tc_pair.cu: two CTAs (cta_group::2) share the X tile of the union of two adjacent CTA tiles' lists
-bool tc_pair_supported(const Geometry &g, int64_t ncols);
-cudaError_t launch_spmm_tc_pair(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
-                                const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy,
-                                int y_dtype, cudaStream_t st);
-
+// `h->plan` is reused when the operands, shape and epilogue are those of the previous call; `h->last` is filled in.
+cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols,
+                           void *d_y, int64_t ldy, int y_dtype, const ConvGeom *conv, cudaStream_t st);
 // spmm_direct.cu
 cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, const uint16_t *d_x, int64_t ldx, int64_t ncols,

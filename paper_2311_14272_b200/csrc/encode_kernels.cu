@@ -47,14 +47,14 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
                     uint32_t *__restrict__ idx, uint8_t *__restrict__ image, uint32_t a_bytes,
                     uint32_t entry_bytes, WalkArgs walks) {
     extern __shared__ uint32_t s_buf[];
-    // The first walks.npairs CTAs build the walk lists of the tensor-core kernel instead of encoding a block:
+    // The first walks.nctas CTAs build the walk lists of the tensor-core kernel instead of encoding a block:
     // that needs only the mask's block list, so it overlaps the encoding instead of following it.
-    if ((int)blockIdx.x < walks.npairs) {
+    if ((int)blockIdx.x < walks.nctas) {
         __shared__ WalkShared s_walks;
         build_walks_body(g, walks, blockIdx.x, s_walks);
         return;
     }
-    const int blk = (int)blockIdx.x - walks.npairs;   // rt * kkeep + slot
+    const int blk = (int)blockIdx.x - walks.nctas;   // rt * kkeep + slot
     const int rt = blk / g.kkeep;
     const int jb = mask_blk_col[blk];
     const int groups = g.bk / M;
@@ -200,7 +200,7 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
             if (e != cudaSuccess) return e;                                                                  \
         }                                                                                                    \
-        kern<<<nblocks + wa.npairs, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits, d_blk_col, \
+        kern<<<nblocks + wa.nctas, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits, d_blk_col, \
                                                      d_vals, d_idx, d_image, a_bytes, entry_bytes, wa);      \
     } while (0)
     if (g.m == 4) {

@@ -324,6 +324,10 @@ cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, i
         group_select_kernel<8><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
 
     const size_t smem = (size_t)g.nblk * (sizeof(unsigned long long) + sizeof(int));
+    if (smem + 64 > 48 * 1024) {     // the longest rows (nblk near 4096) need the opt-in shared-memory size
+        e = cudaFuncSetAttribute(block_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
     block_select_kernel<<<dim3((unsigned)g.nrt, (unsigned)(g.bm / 32)), 256, smem, st>>>(g, score, d_blk_col, d_nm_bits);
     return cudaGetLastError();
 }

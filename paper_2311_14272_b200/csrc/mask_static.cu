@@ -9,8 +9,6 @@
 // fixed-size device array below, which is part of the library image: every GPU that loads the
 // library carries these CRISP_STATIC_SCRATCH_BYTES until the process exits, whether or not
 // this entry point is ever used.
-#include <mutex>
-
 #include "crisp_internal.h"
 
 namespace {
@@ -19,21 +17,13 @@ namespace {
 // address; the address a kernel can use comes from cudaGetSymbolAddress (below).
 static __device__ __align__(256) unsigned char g_static_scratch[CRISP_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
-std::mutex g_lock;
-void *g_scratch_ptr[kMaxDevices] = {};
-
-// Device address of g_static_scratch on the current device, looked up once per device.
+// Device address of g_static_scratch on the current device.  Asked for at every call: the lookup is cheap
+// once the library's module is loaded on the device (the first call loads it), and an address kept
+// across calls would go stale after cudaDeviceReset or in a second context on the same device.
 crisp_status_t scratch_for_current_device(void **out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CRISP_CUDA_ERROR;
-    std::lock_guard<std::mutex> guard(g_lock);
-    if (!g_scratch_ptr[dev]) {
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return CRISP_CUDA_ERROR;
-        g_scratch_ptr[dev] = p;
-    }
-    *out = g_scratch_ptr[dev];
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return CRISP_CUDA_ERROR;
+    *out = p;
     return CRISP_OK;
 }
 

@@ -12,7 +12,8 @@
 // microseconds, is exact, and has no data-dependent control flow.
 #include <climits>
 #include <cmath>
-#include <vector>
+#include <memory>
+#include <new>
 
 #include "crisp_internal.h"
 
@@ -255,7 +256,14 @@ CRISP_API crisp_status_t crisp_global_rank(int32_t n_layers, const crisp_rank_la
     if (s != CRISP_OK) return s;
     if (!d_workspace || !d_kkeep || reinterpret_cast<uintptr_t>(d_workspace) % crisp::kAlign) return CRISP_INVALID_ARG;
     if (!(prune_fraction >= 0.0 && prune_fraction <= 1.0)) return CRISP_INVALID_ARG;
-    std::vector<RankLayer> table((size_t)n_layers);
+    cudaStream_t st = (cudaStream_t)stream;
+    // The layer table is staged from a temporary host array, so the call cannot be part of a stream capture
+    // (the graph would keep a pointer to memory that is gone when it is replayed).
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) return CRISP_CUDA_ERROR;
+    if (cap != cudaStreamCaptureStatusNone) return CRISP_UNSUPPORTED;
+    std::unique_ptr<RankLayer[]> table(new (std::nothrow) RankLayer[(size_t)n_layers]);
+    if (!table) return CRISP_CUDA_ERROR;
     double total = 0.0;
     int off = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -271,13 +279,12 @@ CRISP_API crisp_status_t crisp_global_rank(int32_t n_layers, const crisp_rank_la
         total += (double)L.nrt * (double)L.nblk * (double)L.block_elems;
     }
     const unsigned long long target = (unsigned long long)floor(prune_fraction * total + 0.5);
-    cudaStream_t st = (cudaStream_t)stream;
     uint8_t *ws = reinterpret_cast<uint8_t *>(d_workspace);
     RankLayer *d_table = reinterpret_cast<RankLayer *>(ws + lay.table_off);
     int32_t *d_pruned = reinterpret_cast<int32_t *>(ws + lay.pruned_off);
     RankEntry *d_entries = reinterpret_cast<RankEntry *>(ws + lay.entries_off);
     // the table is read from pageable host memory: the call returns once it has been staged
-    if (cudaMemcpyAsync(d_table, table.data(), table.size() * sizeof(RankLayer), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    if (cudaMemcpyAsync(d_table, table.get(), (size_t)n_layers * sizeof(RankLayer), cudaMemcpyHostToDevice, st) != cudaSuccess)
         return CRISP_CUDA_ERROR;
     if (cudaMemsetAsync(d_pruned, 0, (size_t)n_layers * sizeof(int32_t), st) != cudaSuccess) return CRISP_CUDA_ERROR;
     crisp::rank_columns_kernel<<<n_layers, crisp::kRankThreads, 0, st>>>(d_table, d_entries);

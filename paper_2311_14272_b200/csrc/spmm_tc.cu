@@ -15,6 +15,9 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <atomic>
+#include <new>
+
 #include "crisp_internal.h"
 #include "tc_common.cuh"
 #include "walks.cuh"
@@ -58,6 +61,9 @@ struct TcParams {
     int stack;
     const float *bias;          // layer epilogue: Y = act(W*X + bias); nullptr = no bias
     int relu;
+    unsigned long long wait_limit;   // cycles after which a wait gives up and the kernel reports CRISP_TIMEOUT
+    int skip_fill;              // test hook (-1 = off): the producer leaves out the loads of its skip_fill-th pipeline
+                                // fill, so that the wait for it runs into wait_limit
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
 };
@@ -221,13 +227,13 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
     uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
     for (int t = blockIdx.x; t < p.num_tiles && !*a.abort_flag; t += gridDim.x) {
         const int len = a.walk_len[t % p.nst] * p.stack;
-        if (!mbar_wait(a.bar_tempty + 8 * acc, acc_ph ^ 1u, a.abort_flag)) break;
+        if (!mbar_wait(a.bar_tempty + 8 * acc, acc_ph ^ 1u, a.abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t d_tmem = a.tmem_base + acc * kTileN;
         uint32_t accum = 0;
         bool ok = true;
         for (int e = 0; e < len; ++e) {
-            if (!mbar_wait(full, ph, a.abort_flag)) { ok = false; break; }
+            if (!mbar_wait(full, ph, a.abort_flag, p.wait_limit)) { ok = false; break; }
             tc_fence_after();
             const uint64_t ad = a_desc0 + off, bd = b_desc0 + off;
             if constexpr (kSparse) {
@@ -328,6 +334,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             const uint32_t entry_rows = p.entry_bytes >> 8;      // image rows (256 bytes) per walk entry
             const bool tiled = p.a_map && p.x_map_3d;
             uint32_t dst = ring, full = bar_full, empty = bar_empty, ph = 0;
+            int fill_no = 0;
             for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
                 const int st = t % p.nst, ct = t / p.nst;
                 const int len = walk_len[st];
@@ -352,8 +359,13 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         const int jb = col_q[u];
                         const int krow = jb * p.bk;
                         if (e + kAhead < len) col_q[u] = cols[e + kAhead];
-                        if (!mbar_wait(empty, ph ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
                         mbar_expect_tx(full, tx_bytes);
+                        if (fill_no++ == p.skip_fill) {
+                            // test hook: this fill's copies are left out, so its `full` barrier never completes
+                            // and the bounded wait of the MMA issuer must end the kernel with CRISP_TIMEOUT
+                            if constexpr (kConv) arow += (int)entry_rows; else if (tiled) arow += (int)entry_rows;
+                        } else
                         if constexpr (kConv) {
                             // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box shifted
                             // by the tap; pixels outside the image read as zero (the convolution's padding)
@@ -426,7 +438,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
             const int st = t % p.nst, ct = t / p.nst;
             int go = 0;                                      // lane 0 waits, the warp follows it
-            if (lane == 0) go = !*abort_flag && mbar_wait(bar_tfull + 8 * acc, acc_ph, abort_flag);
+            if (lane == 0) go = !*abort_flag && mbar_wait(bar_tfull + 8 * acc, acc_ph, abort_flag, p.wait_limit);
             go = __shfl_sync(0xFFFFFFFFu, go, 0);
             if (!go) break;
             tc_fence_after();
@@ -666,18 +678,42 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
     for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = s_tile4[i];
 }
 
+typedef void (*TcKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, TcParams);
+
+constexpr int kMaxDevices = 64;
+
+// One instantiation of the kernel: its entry point, its block size, and the largest dynamic shared memory
+// size opted into so far on each device (the attribute belongs to the function on one device).
+struct TcVariant {
+    TcKernel kern;
+    int threads;
+    std::atomic<size_t> *configured;     // [kMaxDevices]
+};
+
 template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi, bool kConv>
-cudaError_t launch_variant(const CUtensorMap &mx, const CUtensorMap &my, const CUtensorMap &ma, const TcParams &p,
-                           int grid, size_t smem, cudaStream_t st) {
-    auto kern = spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi, kConv>;
-    static size_t configured = 0;                       // largest dynamic shared memory opted into so far
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
-    kern<<<grid, 64 + 32 * kEpi, smem, st>>>(mx, my, ma, p);
-    return cudaGetLastError();
+TcVariant make_variant() {
+    static std::atomic<size_t> configured[kMaxDevices];
+    return TcVariant{spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi, kConv>, 64 + 32 * kEpi, configured};
+}
+
+cudaError_t prepare_variant(const TcVariant &v, int device, size_t smem) {
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (smem <= v.configured[device].load(std::memory_order_relaxed)) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void *>(v.kern),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) v.configured[device].store(smem, std::memory_order_relaxed);
+    return e;
+}
+
+// Multiprocessor count of a device, looked up once per device.
+int sm_count_of(int device) {
+    static std::atomic<int> cache[kMaxDevices];
+    if (device < 0 || device >= kMaxDevices) return 148;
+    int n = cache[device].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 148;
+    cache[device].store(n, std::memory_order_relaxed);
+    return n;
 }
 
 }  // namespace
@@ -784,14 +820,7 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
     L.walk_col_off = 0;
     L.walk_len_off = align_up((size_t)L.nst * L.wcap * sizeof(int32_t) + 4);
     L.image_off = L.walk_len_off + align_up((size_t)L.nst * sizeof(int32_t) + 4);
-    // lists for the CTA-pair kernel: union walk of two adjacent CTA tiles and, per union entry and side,
-    // the index of that side's own walk entry (or -1)
-    L.npairs = (L.nst + 1) / 2;
-    L.pwcap = (int)(2 * (int64_t)L.wcap < g.nblk ? 2 * L.wcap : g.nblk);
-    L.pair_col_off = L.image_off + align_up((size_t)L.stack * L.nst * L.wcap * L.entry_bytes + 16);
-    L.pair_len_off = L.pair_col_off + align_up((size_t)L.npairs * L.pwcap * sizeof(int32_t) + 4);
-    L.pair_src_off = L.pair_len_off + align_up((size_t)L.npairs * sizeof(int32_t) + 4);
-    L.total_bytes = L.pair_src_off + align_up((size_t)L.npairs * L.pwcap * 2 * sizeof(int32_t) + 4);
+    L.total_bytes = L.image_off + align_up((size_t)L.stack * L.nst * L.wcap * L.entry_bytes + 16);
     return L;
 }
 
@@ -799,13 +828,10 @@ WalkArgs tc_walk_args(const Geometry &g, bool sparse, const int32_t *d_blk_col, 
     const TcImageLayout L = tc_image_layout(g, sparse);
     WalkArgs a;
     a.blk_col = d_blk_col;
-    a.r = L.r; a.nst = L.nst; a.wcap = L.wcap; a.pwcap = L.pwcap;
-    a.npairs = g.nrt * g.kkeep == 0 ? 0 : L.npairs;
+    a.r = L.r; a.nst = L.nst; a.wcap = L.wcap;
+    a.nctas = g.nrt * g.kkeep == 0 ? 0 : L.nst;
     a.walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
     a.walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
-    a.pair_col = reinterpret_cast<int32_t *>(d_exec + L.pair_col_off);
-    a.pair_len = reinterpret_cast<int32_t *>(d_exec + L.pair_len_off);
-    a.pair_src = reinterpret_cast<int32_t *>(d_exec + L.pair_src_off);
     return a;
 }
 
@@ -817,7 +843,7 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
     int32_t *walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
     int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
     uint8_t *image = d_exec + L.image_off;
-    if (!walks_done) build_walks_kernel<<<L.npairs, 256, 0, st>>>(g, tc_walk_args(g, sparse, d_blk_col, d_exec));
+    if (!walks_done) build_walks_kernel<<<L.nst, 256, 0, st>>>(g, tc_walk_args(g, sparse, d_blk_col, d_exec));
     if (tiles_done) return cudaGetLastError();       // the encode kernel already wrote the weight tiles
     const int grid = L.stack * L.nst * L.wcap;
     const size_t smem_img = (size_t)L.entry_bytes + (size_t)g.vals_per_block() * 2 + (size_t)(g.vals_per_block() * g.idx_bits / 32) * 4 + 16;
@@ -842,17 +868,42 @@ bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int 
            (ldx * 2) % 16 == 0 && (ldy * ye) % 16 == 0 && ncols < (1ll << 31) && encode_tiled_fn() != nullptr;
 }
 
-cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec, int32_t *d_status,
-                           const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y, int64_t ldy, int y_dtype,
-                           int nt_override, const ConvGeom *conv, const Epilogue &epilogue, cudaStream_t st) {
+// Everything one launch needs, and the operands it was planned for.  Encoding three tensor maps costs a few
+// microseconds of host time per call, which small layers notice; a product on the same buffers reuses the plan.
+struct TcPlan {
+    // key
+    const void *x, *y, *bias;
+    int64_t ldx, ldy, ncols;
+    int y_dtype, relu, nt_override, device, skip_stage;
+    unsigned long long wait_limit;
+    bool has_conv;
+    ConvGeom conv;
+    // plan
+    CUtensorMap mx, my, ma;
+    TcParams p;
+    TcVariant variant;
+    int grid;
+    size_t smem;
+    crisp_launch_info_t info;
+};
+
+void tc_plan_destroy(TcPlan *plan) { delete plan; }
+
+namespace {
+
+bool same_conv(const ConvGeom &a, const ConvGeom &b) {
+    return a.batch == b.batch && a.height == b.height && a.width == b.width && a.channels == b.channels &&
+           a.kh == b.kh && a.kw == b.kw && a.pad == b.pad;
+}
+
+// Tile shape, shared-memory split, tensor maps and kernel variant for one product.
+cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y,
+                      int64_t ldy, int y_dtype, const ConvGeom *conv, int device, TcPlan *plan) {
+    const Geometry &g = h->g;
+    const uint8_t *d_exec = h->d_exec;
+    const int nt_override = h->nt_override;
     const TcImageLayout L = tc_image_layout(g, sparse);
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (sm_count <= 0) sm_count = 148;
-    }
+    const int sm_count = sm_count_of(device);
     // column tile: 4 boxes (256 columns).  For the sparse image that leaves room for one accumulator
     // only (256 + 8 metadata columns), which still beats 3 boxes with two accumulators: the kernel is
     // bound by bytes into shared memory, and wider tiles amortise the weight tile over more columns.
@@ -901,8 +952,10 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     p.image = d_exec + L.image_off;
     p.walk_col = reinterpret_cast<const int32_t *>(d_exec + L.walk_col_off);
     p.walk_len = reinterpret_cast<const int32_t *>(d_exec + L.walk_len_off);
-    p.status = d_status;
-    p.bias = epilogue.bias; p.relu = epilogue.relu;
+    p.status = h->d_status;
+    p.bias = h->epilogue.bias; p.relu = h->epilogue.relu;
+    p.wait_limit = h->wait_limit_cycles ? h->wait_limit_cycles : kWaitLimitCycles;
+    p.skip_fill = h->debug_skip_stage;
     p.stack = stack;
     p.nst = L.nst; p.wcap = L.wcap; p.bk = g.bk; p.rows = g.rows; p.ncols = ncols; p.y = d_y; p.ldy = ldy;
     p.n_col_tiles = (int)((ncols + stack * nt * kBoxN - 1) / (stack * nt * kBoxN));
@@ -933,10 +986,10 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
     if (left >= 3 * unit) { p.stg_bufs = 2; p.stg_tile_bytes = 2 * kWideStageBytes; }
     else if (left >= unit) { p.stg_bufs = 2; p.stg_tile_bytes = kWideStageBytes; }
     else { p.stg_bufs = 1; p.stg_tile_bytes = kWideStageBytes; }
-    const size_t smem = (size_t)stages * p.stage_bytes + (size_t)epi * p.stg_bufs * p.stg_tile_bytes + 256 +
-                        (p.walk_cache ? cache_bytes : 0);
+    plan->smem = (size_t)stages * p.stage_bytes + (size_t)epi * p.stg_bufs * p.stg_tile_bytes + 256 +
+                 (p.walk_cache ? cache_bytes : 0);
 
-    CUtensorMap mx, my, ma;
+    CUtensorMap &mx = plan->mx, &my = plan->my, &ma = plan->ma;
     p.a_map = make_map_image(&ma, p.image, (uint64_t)L.stack * L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
     if (!p.a_map) ma = CUtensorMap{};
     const bool f32 = y_dtype != 0;
@@ -950,8 +1003,8 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
         // activation [batch][height][width][channels] and Y [rows][batch][ho][wo] as 4-D tensors
         if (!p.a_map) return cudaErrorInvalidValue;
         p.x_map_3d = 0;
-        const uint64_t c = (uint64_t)conv->channels, w = (uint64_t)conv->width, h = (uint64_t)conv->height;
-        const uint64_t xd[4] = {c, w, h, (uint64_t)conv->batch}, xs[3] = {c * 2, w * c * 2, h * w * c * 2};
+        const uint64_t c = (uint64_t)conv->channels, w = (uint64_t)conv->width, hh = (uint64_t)conv->height;
+        const uint64_t xd[4] = {c, w, hh, (uint64_t)conv->batch}, xs[3] = {c * 2, w * c * 2, hh * w * c * 2};
         const uint32_t xb[4] = {(uint32_t)g.bk, (uint32_t)p.cv_tw, (uint32_t)p.cv_th, (uint32_t)p.cv_tb};
         if (!make_map_4d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_x, xd, xs, xb)) return cudaErrorInvalidValue;
         const uint64_t es = f32 ? 4 : 2, wo = (uint64_t)conv->wo, ho = (uint64_t)conv->ho;
@@ -970,38 +1023,86 @@ cudaError_t launch_spmm_tc(const Geometry &g, bool sparse, const uint8_t *d_exec
                          (uint64_t)ncols, (uint64_t)g.rows, (uint64_t)ldy, f32 ? 32 : 64, p.stg_tile_bytes / 128))
             return cudaErrorInvalidValue;
     }
-    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    plan->grid = (int)(tiles < sm_count ? tiles : sm_count);
+    plan->p = p;
 
-#define CRISP_TC_LAUNCH_C(NTV, SP, ACC, EPI, CONV)                                                        \
-    (f32 ? launch_variant<NTV, SP, ACC, float, EPI, CONV>(mx, my, ma, p, grid, smem, st)                      \
-         : launch_variant<NTV, SP, ACC, uint16_t, EPI, CONV>(mx, my, ma, p, grid, smem, st))
-#define CRISP_TC_LAUNCH_E(NTV, SP, ACC, EPI) CRISP_TC_LAUNCH_C(NTV, SP, ACC, EPI, false)
-#define CRISP_TC_LAUNCH(NTV, SP, ACC) CRISP_TC_LAUNCH_E(NTV, SP, ACC, 8)
+    int acc = 2;
+#define CRISP_TC_VARIANT_C(NTV, SP, ACC, EPI, CONV)                                                       \
+    (acc = ACC, f32 ? make_variant<NTV, SP, ACC, float, EPI, CONV>() : make_variant<NTV, SP, ACC, uint16_t, EPI, CONV>())
+#define CRISP_TC_VARIANT_E(NTV, SP, ACC, EPI) CRISP_TC_VARIANT_C(NTV, SP, ACC, EPI, false)
+#define CRISP_TC_VARIANT(NTV, SP, ACC) CRISP_TC_VARIANT_E(NTV, SP, ACC, 8)
     if (conv) {                              // the gather uses 128- or 256-pixel tiles only
         if (sparse) {
-            if (nt == 2) return CRISP_TC_LAUNCH_C(2, true, 2, 8, true);
-            return epi == 16 ? CRISP_TC_LAUNCH_C(4, true, 1, 16, true) : CRISP_TC_LAUNCH_C(4, true, 1, 8, true);
+            if (nt == 2) plan->variant = CRISP_TC_VARIANT_C(2, true, 2, 8, true);
+            else plan->variant = epi == 16 ? CRISP_TC_VARIANT_C(4, true, 1, 16, true) : CRISP_TC_VARIANT_C(4, true, 1, 8, true);
+        } else {
+            if (nt == 2) plan->variant = CRISP_TC_VARIANT_C(2, false, 2, 8, true);
+            else plan->variant = epi == 16 ? CRISP_TC_VARIANT_C(4, false, 2, 16, true) : CRISP_TC_VARIANT_C(4, false, 2, 8, true);
         }
-        if (nt == 2) return CRISP_TC_LAUNCH_C(2, false, 2, 8, true);
-        return epi == 16 ? CRISP_TC_LAUNCH_C(4, false, 2, 16, true) : CRISP_TC_LAUNCH_C(4, false, 2, 8, true);
-    }
-    if (sparse) {
+    } else if (sparse) {
         switch (nt) {
-            case 1: return CRISP_TC_LAUNCH(1, true, 2);
-            case 2: return CRISP_TC_LAUNCH(2, true, 2);
-            case 3: return epi == 12 ? CRISP_TC_LAUNCH_E(3, true, 2, 12) : CRISP_TC_LAUNCH(3, true, 2);
-            default: return epi == 16 ? CRISP_TC_LAUNCH_E(4, true, 1, 16) : CRISP_TC_LAUNCH(4, true, 1);
+            case 1: plan->variant = CRISP_TC_VARIANT(1, true, 2); break;
+            case 2: plan->variant = CRISP_TC_VARIANT(2, true, 2); break;
+            case 3: plan->variant = epi == 12 ? CRISP_TC_VARIANT_E(3, true, 2, 12) : CRISP_TC_VARIANT(3, true, 2); break;
+            default: plan->variant = epi == 16 ? CRISP_TC_VARIANT_E(4, true, 1, 16) : CRISP_TC_VARIANT(4, true, 1); break;
+        }
+    } else {
+        switch (nt) {
+            case 1: plan->variant = CRISP_TC_VARIANT(1, false, 2); break;
+            case 2: plan->variant = CRISP_TC_VARIANT(2, false, 2); break;
+            case 3: plan->variant = CRISP_TC_VARIANT(3, false, 2); break;
+            default: plan->variant = epi == 16 ? CRISP_TC_VARIANT_E(4, false, 2, 16) : CRISP_TC_VARIANT(4, false, 2); break;
         }
     }
-    switch (nt) {
-        case 1: return CRISP_TC_LAUNCH(1, false, 2);
-        case 2: return CRISP_TC_LAUNCH(2, false, 2);
-        case 3: return CRISP_TC_LAUNCH(3, false, 2);
-        default: return epi == 16 ? CRISP_TC_LAUNCH_E(4, false, 2, 16) : CRISP_TC_LAUNCH(4, false, 2);
+#undef CRISP_TC_VARIANT
+#undef CRISP_TC_VARIANT_E
+#undef CRISP_TC_VARIANT_C
+    crisp_launch_info_t &info = plan->info;
+    info.path = sparse ? CRISP_PATH_SPARSE : CRISP_PATH_DENSE;
+    info.tile_cols = nt * kBoxN;
+    info.accumulators = acc;
+    info.stack = stack;
+    info.epilogue_warps = plan->variant.threads / 32 - 2;
+    info.stages = (int)stages;
+    info.ctas = plan->grid;
+    info.conv = conv ? 1 : 0;
+    return prepare_variant(plan->variant, device, plan->smem);
+}
+
+}  // namespace
+
+cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols,
+                           void *d_y, int64_t ldy, int y_dtype, const ConvGeom *conv, cudaStream_t st) {
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return e;
+    TcPlan *plan = h->plan;
+    const bool hit = plan && plan->x == d_x && plan->y == d_y && plan->ldx == ldx && plan->ldy == ldy &&
+                     plan->ncols == ncols && plan->y_dtype == y_dtype && plan->bias == h->epilogue.bias &&
+                     plan->relu == h->epilogue.relu && plan->nt_override == h->nt_override &&
+                     plan->device == device && plan->skip_stage == h->debug_skip_stage &&
+                     plan->wait_limit == h->wait_limit_cycles && plan->has_conv == (conv != nullptr) &&
+                     (!conv || same_conv(plan->conv, *conv)) && plan->p.status == h->d_status &&
+                     plan->info.path == (sparse ? CRISP_PATH_SPARSE : CRISP_PATH_DENSE);
+    if (!hit) {
+        if (!plan) {
+            plan = new (std::nothrow) TcPlan;
+            if (!plan) return cudaErrorMemoryAllocation;
+            h->plan = plan;
+        }
+        plan->x = nullptr;                                  // not valid until the plan below is complete
+        e = make_plan(h, sparse, d_x, ldx, ncols, d_y, ldy, y_dtype, conv, device, plan);
+        if (e != cudaSuccess) return e;
+        plan->x = d_x; plan->y = d_y; plan->bias = h->epilogue.bias;
+        plan->ldx = ldx; plan->ldy = ldy; plan->ncols = ncols;
+        plan->y_dtype = y_dtype; plan->relu = h->epilogue.relu; plan->nt_override = h->nt_override;
+        plan->device = device; plan->skip_stage = h->debug_skip_stage; plan->wait_limit = h->wait_limit_cycles;
+        plan->has_conv = conv != nullptr;
+        if (conv) plan->conv = *conv;
     }
-#undef CRISP_TC_LAUNCH
-#undef CRISP_TC_LAUNCH_E
-#undef CRISP_TC_LAUNCH_C
+    plan->variant.kern<<<plan->grid, plan->variant.threads, plan->smem, st>>>(plan->mx, plan->my, plan->ma, plan->p);
+    h->last = plan->info;
+    return cudaGetLastError();
 }
 
 }  // namespace crisp

@@ -13,9 +13,6 @@ namespace tc {
 
 constexpr int kTileM = 128;                 // rows per CTA tile = MMA M
 constexpr int kBoxN = 64;                   // columns per TMA box of X (128 bytes, one swizzle span)
-constexpr int kThreads = 192;               // warp 0 producer, warp 1 MMA issuer, warps 2..5 epilogue
-constexpr int kEpiWarps = 4;
-constexpr uint32_t kStageTileBytes = 4096;  // one epilogue staging tile: 32 rows x 128 bytes
 constexpr uint32_t kMetaBytes = 2048;       // 128 rows x 16 bytes of 2:4 metadata per kept block
 constexpr uint32_t kSmemBudget = 232448 - 1024;
 constexpr unsigned long long kWaitLimitCycles = 4000000000ull;   // ~2 s: then report CRISP_TIMEOUT
@@ -44,15 +41,16 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
-// Bounded wait: gives up after kWaitLimitCycles or when another role has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// Bounded wait: gives up after `limit` cycles or when another role has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 0u) {
             if (*abort_flag) return false;
-            if ((unsigned long long)(clock64() - t0) > kWaitLimitCycles) { *abort_flag = 1; return false; }
+            if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return false; }
         }
     }
 }

@@ -78,3 +78,21 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(FileNotFoundError):
         B.load(str(tmp_path / "libcrisp.so"))
+
+
+def test_block_count_limit_per_row_tile(lib):
+    """Up to 4096 k-blocks per row tile are accepted (the longest row the selection kernels hold on chip),
+    one more is refused on the host, before any launch."""
+    ok = B.make_desc(32, 4096 * 32, 2, 4, 32, 32, 0.5)
+    assert B.crisp_keep_count(ok) == (4096, 2048)
+    B.crisp_mask_sizes(ok)
+    with pytest.raises(B.CrispError) as ei:
+        B.crisp_keep_count(B.make_desc(32, 4097 * 32, 2, 4, 32, 32, 0.5))
+    assert ei.value.code == B.UNSUPPORTED
+
+
+def test_handle_queries_reject_null(lib):
+    info = B.LaunchInfo()
+    assert lib.crisp_last_launch(None, C.byref(info)) == B.INVALID_ARG
+    assert lib.crisp_set_tuning(None, 0, 0, -1) == B.INVALID_ARG
+    assert lib.crisp_reset_status(None, None) == B.INVALID_ARG

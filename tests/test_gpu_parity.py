@@ -45,10 +45,11 @@ CASES = [
     (64, 96, 50, 8, 8, 32, 32, 0.67),
     (130, 384, 96, 2, 4, 128, 128, 0.34),
     (64, 288, 40, 3, 8, 64, 96, 0.67),
-    (384, 768, 576, 2, 4, 128, 64, 0.5),     # 3 CTA tiles (odd: one pair has a ghost side), 2.25 column tiles
+    (384, 768, 576, 2, 4, 128, 64, 0.5),     # 3 CTA tiles, 2.25 column tiles
     (512, 512, 320, 1, 4, 64, 64, 0.25),
     (256, 256, 128, 2, 8, 32, 32, 0.5),
-    # thin layers (one CTA tile of at most 32 / 64 rows): a tile covers 4 / 2 column tiles, one per lane group
+    # thin layers (one CTA tile of at most 32 / 64 rows) with few columns: too few tiles for the stacked
+    # accumulator, so these run the ordinary tiles (the stacked path has its own cases below)
     (16, 32, 5000, 2, 8, 32, 32, 1.0),
     (24, 96, 3000, 2, 8, 32, 32, 0.67),
     (32, 192, 4100, 2, 4, 32, 64, 0.5),
@@ -59,25 +60,23 @@ CASES = [
 
 # which execution image crisp_encode lays out: the default choice (2:4 sparse MMA when n <= 2, dense
 # tiles otherwise), dense tiles forced, or none (CUDA-core kernel on the canonical format)
-# "pair" / "dense-pair": same images, run by the CTA-pair kernel where the shape allows it
-IMAGES = ["auto", "dense", "none", "pair", "dense-pair"]
+IMAGES = ["auto", "dense", "none"]
 
 
 @pytest.fixture(params=IMAGES)
 def image(request, monkeypatch):
     kind = request.param
-    monkeypatch.setenv("CRISP_TC_PAIR", "1" if kind.endswith("pair") else "0")
-    if kind in ("auto", "pair"):
+    if kind == "auto":
         monkeypatch.delenv("CRISP_EXEC_IMAGE", raising=False)
     else:
-        monkeypatch.setenv("CRISP_EXEC_IMAGE", "dense" if kind.startswith("dense") else kind)
+        monkeypatch.setenv("CRISP_EXEC_IMAGE", kind)
     return kind
 
 
 def expected_path(B, image, n, kkeep=1):
     if image == "none":
         return B.PATH_DIRECT
-    if image.startswith("dense"):
+    if image == "dense":
         return B.PATH_DENSE
     return B.PATH_SPARSE if n <= 2 else B.PATH_DENSE
 
@@ -101,6 +100,7 @@ def test_layer_matches_oracle(env, image, rows, k, ncols, n, m, bm, bk, keep, y_
     L.spmm(xbuf[:, :ncols], y=ybuf[:, :ncols], y_dtype=y_dtype)
     torch.cuda.synchronize()
     assert L.device_status() == 0
+    assert L.last_launch()["path"] == expected_path(B, image, n)          # the kernel family that really ran
     check_tolerance(y_to_f64(ybuf[:, :ncols], torch), oracle.spmm_fp64(wd, x))
     assert torch.all(ybuf[:, ncols:] == 5.0)                             # nothing written past ncols
     L.close()
@@ -136,6 +136,9 @@ def test_padded_leading_dimensions_and_odd_alignment(env):
     xbuf[:, :90] = bf16_dev(x, torch)
     ybuf = torch.full((100, 101), 7.0, dtype=torch.bfloat16, device="cuda")
     L.spmm(xbuf[:, :90], y=ybuf[:, :90])
+    # pitches of 97 and 101 elements are not multiples of 16 bytes: TMA cannot address them, and the call
+    # must have fallen back to the CUDA-core kernel although the handle carries a tensor-core image
+    assert L.bytes_model(90)["path"] == B.PATH_SPARSE and L.last_launch()["path"] == B.PATH_DIRECT
     check_tolerance(y_to_f64(ybuf[:, :90], torch), oracle.spmm_fp64(wd, x))
     assert torch.all(ybuf[:, 90:] == 7.0)                                # nothing written past ncols
 
@@ -219,3 +222,94 @@ def test_config2_full(env, image):
     full = oracle.spmm_fp64_skipzero(wd, x)                               # shown equal on small shapes
     assert np.array_equal(full[sel], ref_rows)
     check_tolerance(y_to_f64(y, torch), full)
+
+
+# Thin layers with enough columns for the stacked accumulator: one accumulator covers `stack` column tiles,
+# one per group of 128 / stack lanes, and the walk is repeated per group against that group's columns.
+# ncols is chosen so that there are at least as many stacked tiles as SMs (148) plus a ragged tail.
+STACKED = [
+    # rows, k, n, m, bm, bk, keep, ncols, stack
+    (16, 32, 2, 8, 32, 32, 1.0, 148 * 4 * 256 + 1000, 4),
+    (32, 64, 2, 4, 32, 32, 1.0, 148 * 4 * 192 + 520, 4),       # two-block walk: 192-column tiles, two accumulators
+    (64, 64, 2, 8, 32, 32, 1.0, 148 * 2 * 256 + 776, 2),       # two row tiles of 32 in a 64-row window
+    (48, 128, 1, 4, 64, 64, 0.5, 148 * 2 * 256 + 264, 2),      # 48 of 64 rows, one kept block of two
+    (40, 64, 3, 4, 64, 64, 1.0, 148 * 2 * 256 + 128, 2),       # dense-tile image
+]
+
+
+@pytest.mark.parametrize("rows,k,n,m,bm,bk,keep,ncols,stack", STACKED)
+@pytest.mark.parametrize("y_dtype", [0, 1])
+@pytest.mark.parametrize("epilogue", [False, True])
+def test_stacked_thin_layer_matches_oracle(env, rows, k, n, m, bm, bk, keep, ncols, stack, y_dtype, epilogue):
+    B, torch = env
+    w, s, x = rand_inputs(rows, k, ncols, seed=rows * 7 + k + stack)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
+    L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)
+    ref = oracle.spmm_fp64(wd, x)
+    if epilogue:
+        bias = np.random.default_rng(rows).standard_normal(rows).astype(np.float32)
+        L.set_epilogue(to_dev(bias, torch), relu=True)
+        ref = oracle.bias_relu(ref, bias, True)
+    y = L.spmm(bf16_dev(x, torch), y_dtype=y_dtype)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    info = L.last_launch()
+    assert info["stack"] == stack, info                       # the stacked path is the one that ran
+    assert info["path"] == (B.PATH_SPARSE if n <= 2 else B.PATH_DENSE)
+    check_tolerance(y_to_f64(y, torch), ref)
+    L.close()
+
+
+def test_identity_activation_wide_single_accumulator_tile(env):
+    """The launch configuration of the large layers (256-column tiles, sparse image, one accumulator) on
+    X = [I I I ...]: column c of Y must be column c mod k of the decoded weight, bit for bit."""
+    B, torch = env
+    rows, k, n, m, bm, bk, keep = 256, 256, 2, 4, 128, 64, 0.5
+    ncols = 148 * 256 // 2 + 256                              # enough tiles that the column tile is not narrowed
+    w, s, _ = rand_inputs(rows, k, 8, seed=99)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
+    L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
+    eye = torch.eye(k, dtype=torch.bfloat16, device="cuda").repeat(1, ncols // k)
+    y = L.spmm(eye)
+    torch.cuda.synchronize()
+    info = L.last_launch()
+    assert info["path"] == B.PATH_SPARSE and info["tile_cols"] == 256 and info["accumulators"] == 1, info
+    got = wl.bf16_bits_to_f32(y.view(torch.int16).cpu().numpy().view(np.uint16))
+    want = np.tile(wl.bf16_bits_to_f32(wb), (1, ncols // k))
+    assert np.array_equal(got, want)
+    assert L.device_status() == 0
+
+
+def test_bounded_wait_reports_timeout_and_the_handle_stays_usable(env):
+    """Failure detection: a pipeline fill whose copies never arrive must end the kernel through its bounded
+    waits (status CRISP_TIMEOUT), and the next product on the same handle and stream must be correct."""
+    B, torch = env
+    rows, k, ncols, n, m, bm, bk, keep = 128, 256, 512, 2, 4, 128, 64, 0.5
+    w, s, x = rand_inputs(rows, k, ncols, seed=4242)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
+    L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
+    d_x = bf16_dev(x, torch)
+    L.set_tuning(wait_limit_cycles=2_000_000, skip_fill=1)    # about a millisecond
+    L.spmm(d_x)
+    torch.cuda.synchronize()
+    assert L.device_status() == B.TIMEOUT
+    L.set_tuning()                                            # defaults again
+    L.reset_status()
+    y = L.spmm(d_x)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    check_tolerance(y_to_f64(y, torch), oracle.spmm_fp64(wd, x))
+
+
+def test_longest_row_of_blocks(env):
+    """4096 k-blocks per row tile: the per-row-tile selection holds a whole row of scores in shared memory
+    (more than the default 48 KB at this length)."""
+    B, torch = env
+    rows, k = 32, 4096 * 32
+    rng = np.random.default_rng(8)
+    s = rng.uniform(0.1, 2.0, (rows, k)).astype(np.float32)
+    w = wl.f32_to_bf16_bits(rng.standard_normal((rows, k)).astype(np.float32))
+    mk, vals, idx, wd, wb = oracle_layer(w, s, 1, 4, 32, 32, 0.3)
+    L = gpu_layer(B, torch, w, s, 1, 4, 32, 32, 0.3)
+    assert_mask_and_encoding_equal(L, mk, vals, idx)

@@ -1,9 +1,10 @@
 """crisp_build_mask_static: the mask projection for callers that are not allowed to allocate
 device memory when they call (plug-ins inside a framework that owns the GPU's memory, loops that
 must stay allocation-free after start-up).  Its scratch is a fixed array inside the library, so
-the test checks three things a user relies on: the result is bit-identical to crisp_build_mask,
-a second call right after the first is not disturbed by what the first left in the shared array,
-and a layer too large for the array is refused instead of overrunning it."""
+the test checks what a user relies on: the result is bit-identical to crisp_build_mask (and to the
+CPU oracle's mask of the same saliency), a second call right after the first is not disturbed by what
+the first left in the shared array, and a layer too large for the array is refused instead of
+overrunning it."""
 import ctypes as C
 
 import numpy as np
@@ -46,6 +47,9 @@ def test_static_scratch_mask_matches_the_workspace_version_twice_in_a_row():
         assert np.array_equal(got_cols, want_cols)        # integer outputs: compared bit for bit,
         assert np.array_equal(got_bits, want_bits)        # the same bar as the other mask tests
         assert want_bits.any()
+        import oracle
+        mk = oracle.build_mask(s, n, m, bm, bk, keep)         # and both agree with the definition
+        assert np.array_equal(got_cols, mk.blk_col) and np.array_equal(got_bits, mk.nm_bits)
     torch.cuda.synchronize()
 
 
