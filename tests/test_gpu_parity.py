@@ -230,7 +230,8 @@ def test_config2_full(env, image):
 STACKED = [
     # rows, k, n, m, bm, bk, keep, ncols, stack
     (16, 32, 2, 8, 32, 32, 1.0, 148 * 4 * 256 + 1000, 4),
-    (32, 64, 2, 4, 32, 32, 1.0, 148 * 4 * 192 + 520, 4),       # two-block walk: 192-column tiles, two accumulators
+    (32, 64, 2, 4, 32, 32, 1.0, 148 * 4 * 256 + 520, 4),       # two blocks, walked once per lane group
+    (64, 32, 2, 8, 32, 32, 1.0, 148 * 2 * 256 + 328, 2),       # one-block walk: 192-column tiles, two accumulators
     (64, 64, 2, 8, 32, 32, 1.0, 148 * 2 * 256 + 776, 2),       # two row tiles of 32 in a 64-row window
     (48, 128, 1, 4, 64, 64, 0.5, 148 * 2 * 256 + 264, 2),      # 48 of 64 rows, one kept block of two
     (40, 64, 3, 4, 64, 64, 1.0, 148 * 2 * 256 + 128, 2),       # dense-tile image
@@ -265,8 +266,8 @@ def test_identity_activation_wide_single_accumulator_tile(env):
     """The launch configuration of the large layers (256-column tiles, sparse image, one accumulator) on
     X = [I I I ...]: column c of Y must be column c mod k of the decoded weight, bit for bit."""
     B, torch = env
-    rows, k, n, m, bm, bk, keep = 256, 256, 2, 4, 128, 64, 0.5
-    ncols = 148 * 256 // 2 + 256                              # enough tiles that the column tile is not narrowed
+    rows, k, n, m, bm, bk, keep = 256, 1024, 2, 4, 128, 64, 0.6     # walks of 10 blocks: the long-walk variant
+    ncols = 19 * k                                            # enough tiles that the column tile is not narrowed
     w, s, _ = rand_inputs(rows, k, 8, seed=99)
     mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
     L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
