@@ -51,6 +51,9 @@ def pick_layer(name: str) -> wl.Layer:
         nm, keep = name[len("sweep_"):].split("_keep")
         n, m = nm.split(":")
         return wl.sweep_cell(int(n), int(m), float(keep))
+    for l in wl.config3() + wl.config4():
+        if l.name == name:
+            return l
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -230,54 +233,126 @@ def roofline_terms(model, peaks, spmm_ms, ncols):
             "frac_literal": max(useful / (peaks["bf16_tflops"] * 1e12), t_hbm) / (spmm_ms * 1e-3)}
 
 
-CELL_WORKLOADS = ["sweep_2:4_keep1.0", "sweep_2:4_keep0.25", "sweep_2:4_keep0.1", "sweep_1:4_keep0.5",
-                  "sweep_2:8_keep0.5", "sweep_4:8_keep0.5", "config2"]
+def all_cells():
+    """Every (config, layer, N:M, keep) the metric names: config 1, config 2, the 13 VGG-16 and the 35
+    MobileNetV2 layers, the 5 x 4 sweep, and 3:4 on the sweep shape."""
+    return wl.config1() + wl.config2() + wl.config3() + wl.config4() + wl.config5() + wl.extra_sweep_cells()
 
 
-def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=12):
-    """SpMM-only timings of further cells of the metric (same protocol: events, L2 flushed between
-    iterations), each beside a dense bf16 cuBLAS GEMM of the same shape."""
+def device_activation(torch, layer, dev):
+    """X[k, ncols] bf16 drawn on the device (N(0,1), rectified for the network layers): the stand-in for the
+    layer's input activations.  Same distribution as workloads.make_activation; the large layers' X (up to
+    0.9 GB) is not worth a host draw and a copy per cell."""
+    g = torch.Generator(device=dev)
+    g.manual_seed(layer.seed + 7)
+    x = torch.randn((layer.k, layer.ncols), device=dev, generator=g)
+    if layer.relu_x:
+        x.clamp_(min=0)
+    return x.to(torch.bfloat16)
+
+
+def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=50):
+    """SpMM-only timing of every cell of the metric, each beside a dense bf16 cuBLAS GEMM of the same shape.
+    Cold L2: `iters` launches, each after an L2 flush, each in its own event pair (median and minimum).
+    Warm L2: the same launch repeated back to back on the same buffers, `iters` launches in five event pairs
+    (median and minimum of the five averages); for layers larger than L2 that is simply a pipelined stream of
+    launches."""
     out = []
     stream = torch.cuda.current_stream()
-    for name in CELL_WORKLOADS:
-        layer = pick_layer(name)
-        if name.startswith("sweep_"):
+
+    def cold(fn):
+        ts = []
+        for i in range(3 + iters):
+            flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b) * 1e3)
+        return float(np.median(ts)), float(np.min(ts))
+
+    def warm(fn):
+        per = max(1, iters // 5)
+        ts = []
+        for _ in range(3):
+            fn()
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(per):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3 / per)
+        return float(np.median(ts)), float(np.min(ts))
+
+    for layer in all_cells():
+        if layer.config == 5:
             d_s, d_w, d_x = shared                      # every sweep cell prunes the same W / S / X
         else:
-            w, s, x = wl.make_layer_inputs(layer)
-            d_s = torch.from_numpy(s).to(dev)
+            w = wl.make_weight(layer)
+            d_s = torch.from_numpy(wl.make_saliency(layer, w)).to(dev)
             d_w = torch.from_numpy(w.view(np.int16)).to(dev).view(torch.bfloat16)
-            d_x = torch.from_numpy(x.view(np.int16)).to(dev).view(torch.bfloat16)
+            d_x = device_activation(torch, layer, dev)
         d_y = torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16, device=dev)
         L = B.HybridLayer(layer.rows, layer.k, layer.n, layer.m, layer.block_rows, layer.block_k,
                           layer.keep_ratio, device=dev)
         L.build_mask(d_s).encode(d_w)
-        ts, td = [], []
-        for i in range(3 + iters):
-            flush_l2()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            L.spmm(d_x, y=d_y)
-            b.record(stream)
-            flush_l2()
-            c, d = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            c.record(stream)
-            torch.matmul(d_w, d_x, out=d_y)
-            d.record(stream)
-            torch.cuda.synchronize()
-            if i >= 3:
-                ts.append(a.elapsed_time(b)); td.append(c.elapsed_time(d))
+        ours = lambda: L.spmm(d_x, y=d_y)
+        dense = lambda: torch.matmul(d_w, d_x, out=d_y)
+        c_med, c_min = cold(ours)
+        w_med, w_min = warm(ours)
+        launched = L.last_launch()
+        dc_med, dc_min = cold(dense)
+        dw_med, dw_min = warm(dense)
         model = L.bytes_model(layer.ncols)
-        ms = float(np.mean(ts))
-        r = roofline_terms(model, peaks, ms, layer.ncols)
-        out.append({"workload": name, "kernel": B.PATH_NAMES[model["path"]], "kkeep": L.kkeep,
-                    "spmm_us": ms * 1e3, "dense_cublas_us": float(np.mean(td)) * 1e3,
-                    "speedup_vs_dense_cublas": float(np.mean(td)) / ms,
-                    "useful_tflops": r["useful_flops"] / (ms * 1e-3) / 1e12,
-                    "t_tensor_us": r["t_tensor"] * 1e6, "t_hbm_us": r["t_hbm"] * 1e6,
-                    "roofline_frac": r["frac"], "roofline_frac_literal": r["frac_literal"],
-                    "device_status": L.device_status()})
+        rec = {"workload": layer.name, "config": layer.config, "rows": layer.rows, "k": layer.k,
+               "ncols": layer.ncols, "nm": f"{layer.n}:{layer.m}", "block": [layer.block_rows, layer.block_k],
+               "keep": round(layer.keep_ratio, 4), "kkeep": L.kkeep, "kernel": B.PATH_NAMES[launched["path"]],
+               "tile_cols": launched["tile_cols"], "accumulators": launched["accumulators"],
+               "stack": launched["stack"],
+               "spmm_us": c_med, "spmm_us_min": c_min, "spmm_warm_us": w_med, "spmm_warm_us_min": w_min,
+               "dense_cublas_us": dc_med, "dense_cublas_us_min": dc_min, "dense_cublas_warm_us": dw_med,
+               "speedup_vs_dense_cublas": dc_med / c_med, "speedup_warm": dw_med / w_med,
+               "device_status": L.device_status()}
+        if L.kkeep > 0:
+            r = roofline_terms(model, peaks, c_med * 1e-3, layer.ncols)
+            rec.update({"useful_tflops": r["useful_flops"] / (c_med * 1e-6) / 1e12,
+                        "t_tensor_us": r["t_tensor"] * 1e6, "t_hbm_us": r["t_hbm"] * 1e6,
+                        "roofline_frac": r["frac"], "roofline_frac_literal": r["frac_literal"],
+                        "roofline_frac_warm": r["frac"] * c_med / w_med})
+        else:
+            # no kept block (a one-block layer below keep 0.5): Y = 0, no useful work, kept out of the sums
+            rec.update({"useful_tflops": 0.0, "roofline_frac": None, "roofline_frac_literal": None})
+        out.append(rec)
         L.close()
+        del d_y
+        if layer.config != 5:
+            del d_x, d_w, d_s
+    return out
+
+
+def summarise_cells(cells):
+    """Per workload family: sum of our times, sum of the dense cuBLAS times, their ratio (layers with no kept
+    block left out), and the spread of the roofline fraction."""
+    fam = {1: "config1", 2: "config2_resnet50_layer3", 3: "config3_vgg16", 4: "config4_mobilenetv2", 5: "config5_sweep"}
+    out = {}
+    for cfg, name in fam.items():
+        cs = [c for c in cells if c["config"] == cfg and c["kkeep"] > 0]
+        if not cs:
+            continue
+        ours, dense = sum(c["spmm_us"] for c in cs), sum(c["dense_cublas_us"] for c in cs)
+        fr = [c["roofline_frac"] for c in cs]
+        out[name] = {"layers": len(cs), "spmm_us_sum": ours, "dense_cublas_us_sum": dense,
+                     "speedup_vs_dense_cublas": dense / ours,
+                     "useful_tflops": sum(c["useful_tflops"] * c["spmm_us"] for c in cs) / ours,
+                     "roofline_frac_min": min(fr), "roofline_frac_median": float(np.median(fr)),
+                     "roofline_frac_max": max(fr),
+                     "faster_than_dense": sum(1 for c in cs if c["speedup_vs_dense_cublas"] >= 1.0)}
+    low = [c for c in cells if c["config"] == 5 and c["keep"] <= 0.5 and c["kkeep"] > 0]
+    out["sweep_keep_le_0.5"] = {"cells": len(low),
+                                "at_or_above_60pct_of_roofline": sum(1 for c in low if c["roofline_frac"] >= 0.6),
+                                "faster_than_dense": sum(1 for c in low if c["speedup_vs_dense_cublas"] >= 1.0)}
     return out
 
 
@@ -607,6 +682,62 @@ def run_ours(args, layer, rank, world):
         dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
     e2e_ms = float(e2e_ms.item())
 
+    # ---- end to end, inference style: the handle (mask + encoding) is reused, a step is X in -> product -> Y out.
+    # Same pipelining: the copy of the next X and the read-back of the previous Y overlap the product.
+    def inf_pipelined(n, start_event):
+        s_in.wait_event(start_event)
+        for it in range(n):
+            k = it & 1
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_cmp[k])
+                d_in[k][2].view(torch.int16).copy_(h_x, non_blocking=True)
+                ev_in[k].record(s_in)
+            stream.wait_event(ev_in[k])
+            stream.wait_event(ev_out[k])
+            L.spmm(d_in[k][2], y=d_out[k])
+            ev_cmp[k].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_cmp[k])
+                h_out[k].copy_(d_out[k], non_blocking=True)
+                ev_out[k].record(s_out)
+        stream.wait_event(ev_out[0])
+        stream.wait_event(ev_out[1])
+
+    L.build_mask(d_s)
+    L.encode(d_w)
+    a = torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    inf_pipelined(2, a)
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    inf_pipelined(e2e_steps, a)
+    b.record(stream)
+    barrier()
+    inf_ms = torch.tensor([a.elapsed_time(b) / e2e_steps], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(inf_ms, op=dist.ReduceOp.MAX)
+    inf_ms = float(inf_ms.item())
+
+    # ---- the SpMM kernel as a stream of launches: back to back on three rotating sets of X / Y (384 MB, larger
+    # than L2, so every launch finds its operands in HBM), one event pair around the whole stream
+    xs = [d_x, d_in[1][2], torch.empty_like(d_x)]
+    xs[1].copy_(d_x); xs[2].copy_(d_x)
+    ys = [d_y, d_out[1], torch.empty_like(d_y)]
+    b2b = []
+    for rep in range(4):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_launch = 18
+        a.record(stream)
+        for i in range(n_launch):
+            L.spmm(xs[i % 3], y=ys[i % 3])
+        b.record(stream)
+        torch.cuda.synchronize()
+        if rep:
+            b2b.append(a.elapsed_time(b) * 1e3 / n_launch)
+    t_b2b_us = float(np.median(b2b))
+    del xs, ys
+
     useful_flops = 2.0 * nnz * layer.ncols
     value = world * useful_flops / (ms_per_step * 1e-3) / 1e12
     e2e_value = world * useful_flops / (e2e_ms * 1e-3) / 1e12
@@ -623,8 +754,17 @@ def run_ours(args, layer, rank, world):
     else:
         roof = {"bound": "hbm", "achieved": hbm_bytes / (spmm_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update({"traffic": recorded_traffic(args.workload, B.PATH_NAMES[model["path"]]), "peak_kind": f"of {peak_kind} (burst)", "kernel": B.PATH_NAMES[model["path"]],
+    launched = L.last_launch()
+    roof.update({"traffic": recorded_traffic(args.workload, B.PATH_NAMES[launched["path"]]), "peak_kind": f"of {peak_kind} (burst)",
+                 "kernel": B.PATH_NAMES[launched["path"]], "tile_cols": launched["tile_cols"],
+                 "accumulators": launched["accumulators"], "ring_stages": launched["stages"], "ctas": launched["ctas"],
                  "t_tensor_us": t_tensor * 1e6, "t_hbm_us": t_hbm * 1e6, "t_kernel_us": spmm_ms * 1e3,
+                 "t_kernel_median_us": float(np.median(t_spmm) * 1e3), "t_kernel_min_us": float(t_spmm.min() * 1e3),
+                 "t_kernel_timing": "mean over the timed steps of the event pair around the crisp_spmm launch (L2 flushed before every step)",
+                 "t_kernel_back_to_back_us": t_b2b_us,
+                 "frac_back_to_back": max(t_tensor, t_hbm) / (t_b2b_us * 1e-6),
+                 "dense_cublas_us": float(t_dense.mean() * 1e3),
+                 "speedup_vs_dense_cublas": float(t_dense.mean() / t_spmm.mean()),
                  "frac_of_max_roof": max(t_tensor, t_hbm) / (spmm_ms * 1e-3),
                  "frac_literal_useful_flops": useful_flops / (spmm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                  "algorithmic_bytes": hbm_bytes, "slot_flops": slot_flops})
@@ -654,11 +794,16 @@ def run_ours(args, layer, rank, world):
                    "overlap": "copies of step i+1 overlap compute and read-back of step i (2 buffer sets, 3 streams)",
                    "h2d_bytes_per_step": int(h_s.numel() * 4 + h_w.numel() * 2 + h_x.numel() * 2),
                    "d2h_bytes_per_step": int(h_y.numel() * 2)},
+           "e2e_inference": {"value": world * useful_flops / (inf_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": inf_ms,
+                             "step": "X host -> device, crisp_spmm on the resident handle, Y device -> host (2 buffer sets, 3 streams)",
+                             "h2d_bytes_per_step": int(h_x.numel() * 2), "d2h_bytes_per_step": int(h_y.numel() * 2)},
            "gpu_launches": sum(kernels_per_step.values()) * args.steps, "kernels_per_step": kernels_per_step,
            "clocks": clocks, "roofline": roof, "phases": phases, "device_status": status}
 
     if rank == 0 and world == 1 and not args.no_cells and args.workload.startswith("sweep_"):
-        out["cells"] = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
+        cells = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x), iters=args.cell_iters)
+        out["summary"] = summarise_cells(cells)
+        out["cells"] = cells
         out["global_rank"] = measure_global_rank(torch, B, dev, not args.no_cpu_baseline)
         out["conv"] = measure_conv(torch, B, dev, peaks, flush_l2)
         out["saliency"] = measure_saliency(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
@@ -683,9 +828,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="sweep_2:4_keep0.5",
-                    help="sweep_<n>:<m>_keep<r> (4096x4096x8192, block 128x64), config1 or config2")
+                    help="sweep_<n>:<m>_keep<r> (4096x4096x8192, block 128x64), config1, config2, or a layer name "
+                         "of config 3 / 4 (vgg16_conv<i>, mbv2_b<i>_expand, mbv2_b<i>_project, mbv2_last)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-cells", action="store_true", help="skip the extra SpMM-only cells")
+    ap.add_argument("--no-cells", action="store_true", help="skip the per-layer / per-cell SpMM timings")
+    ap.add_argument("--cell-iters", type=int, default=50, help="timed launches per cell and protocol")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -179,8 +179,15 @@ def config5(rows: int = 4096, k: int = 4096, ncols: int = 8192) -> List[Layer]:
     return out
 
 
+def extra_sweep_cells(rows: int = 4096, k: int = 4096, ncols: int = 8192) -> List[Layer]:
+    """3:4 on the sweep shape: the third pattern the paper's accelerator supports (Sec. III-D), which the
+    five N:M ratios of the sweep do not contain.  Same W / S / X as the sweep."""
+    return [Layer(5, 0, f"sweep_3:4_keep{keep}", rows, k, ncols, 3, 4, 128, 64, keep, 0.02, False)
+            for keep in SWEEP_KEEP]
+
+
 def sweep_cell(n: int, m: int, keep: float, **kw) -> Layer:
-    for l in config5(**kw):
+    for l in config5(**kw) + extra_sweep_cells(**kw):
         if (l.n, l.m) == (n, m) and abs(l.keep_ratio - keep) < 1e-12:
             return l
     raise KeyError((n, m, keep))
