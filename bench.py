@@ -406,6 +406,54 @@ def measure_global_rank(torch, B, dev, with_oracle, iters=12):
     return out
 
 
+def measure_iteration(torch, B, dev, with_oracle, samples=4, iters=9):
+    """One pruning iteration of Algorithm 1 over a whole network without the fine-tuning (saliency of Eq. 1 from
+    `samples` bf16 gradient tensors per layer, N:M step + block scores, global rank selection, per-row-tile
+    selection, compression), through binding.PruningNetwork: device time of the whole sequence (it contains one
+    small device-to-host read of the selected counts), its launches, and the oracle's time for the same step."""
+    out = []
+    stream = torch.cuda.current_stream()
+    for name, cfg in (("vgg16", wl.config3()), ("mobilenetv2", wl.config4())):
+        n, m, bm, bk = cfg[0].n, cfg[0].m, cfg[0].block_rows, cfg[0].block_k
+        shapes = [(l.rows, l.k) for l in cfg]
+        w_host = [wl.make_weight(l) for l in cfg]
+        g = torch.Generator(device=dev); g.manual_seed(cfg[0].seed + 91)
+        d_w = [torch.from_numpy(w.view(np.int16)).to(dev).view(torch.bfloat16) for w in w_host]
+        d_g = [[(torch.randn(sh, device=dev, generator=g) * 1e-2).to(torch.bfloat16) for _ in range(samples)] for sh in shapes]
+        net = B.PruningNetwork(shapes, n, m, bm, bk, min_keep=1, device=dev)
+        kappa = 1.0 - 0.5 * n / m                                 # half of the blocks of the network
+        ts = []
+        for i in range(3 + iters):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            kk = net.step(d_w, d_g, kappa)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b) * 1e3)
+        weights = sum(r * k for r, k in shapes)
+        rec = {"network": name, "layers": len(shapes), "weights": int(weights), "samples": samples, "kappa": kappa,
+               "iteration_us": float(np.median(ts)), "iteration_us_min": float(np.min(ts)),
+               "launches": len(shapes) * (samples + 2 + 3 + 1 + 2) + 3, "kkeep": [int(c) for c in kk],
+               "algorithmic_bytes": int(weights * (samples * 2 + (samples - 1) * 8 + 4 + 2 + 4 + 4 + 4 + 2 + 2))}
+        rec["achieved_gbs"] = rec["algorithmic_bytes"] / (rec["iteration_us"] * 1e-6) / 1e9
+        if with_oracle:
+            import oracle
+            grads = [np.stack([wl.bf16_bits_to_f32(t.view(torch.int16).cpu().numpy().view(np.uint16)) for t in gs]) for gs in d_g]
+            t0 = time.perf_counter()
+            sal = [oracle.saliency_f32(gr, w) for gr, w in zip(grads, w_host)]
+            full = [oracle.build_mask(s_, n, m, bm, bk, 1.0) for s_ in sal]
+            want = oracle.global_rank([f.score for f in full], [oracle.score_scale_exp(s_) for s_ in sal],
+                                      [bm * bk] * len(full), B.crisp_prune_fraction(kappa, n, m), min_keep=[1] * len(full))
+            for s_, w, f, c in zip(sal, w_host, full, want):
+                oracle.encode(w, oracle.build_mask(s_, n, m, bm, bk, float(c) / f.nblk))
+            rec["oracle_us"] = (time.perf_counter() - t0) * 1e6
+            rec["matches_oracle"] = bool([int(c) for c in want] == rec["kkeep"])
+        net.close()
+        out.append(rec)
+    return out
+
+
 _VGG_CONV = {1: (64, 224), 2: (64, 112), 3: (128, 112)}     # config-3 layer index -> (input channels, side)
 
 
@@ -807,6 +855,7 @@ def run_ours(args, layer, rank, world):
         out["global_rank"] = measure_global_rank(torch, B, dev, not args.no_cpu_baseline)
         out["conv"] = measure_conv(torch, B, dev, peaks, flush_l2)
         out["saliency"] = measure_saliency(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
+        out["pruning_iteration"] = measure_iteration(torch, B, dev, not args.no_cpu_baseline)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)

@@ -142,6 +142,40 @@ CRISP_API crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s,
                                           crisp_mask_t *out);
 
 /*
+ * crisp_build_mask with options.  flags:
+ *   CRISP_MASK_MAX_KNOWN  the first word of d_workspace already holds the bits of the layer's largest
+ *                         canonical |s| (crisp_saliency_finish_max wrote it while it produced d_saliency):
+ *                         the pass over the saliency that finds that maximum is skipped.  A wrong value gives
+ *                         a wrong fixed-point scale, i.e. a different (still valid) block ranking.
+ * flags = 0 is crisp_build_mask.
+ */
+#define CRISP_MASK_MAX_KNOWN 1u
+CRISP_API crisp_status_t crisp_build_mask_ex(const float *d_saliency, int64_t ld_s,
+                                             const crisp_layer_desc_t *desc, void *d_mask_buf,
+                                             void *d_workspace, uint32_t flags, void *stream,
+                                             crisp_mask_t *out);
+
+/*
+ * Keep fewer blocks of an existing mask without streaming the saliency again: the per-row-tile selection of
+ * Algorithm 1 (sort per row, select, prune) re-run on the block scores and group bits that the mask's
+ * crisp_build_mask left in d_workspace and d_mask_buf.  kkeep must not exceed the mask's current count
+ * (the kept sets of one ranking are nested; INVALID_ARG otherwise).  Afterwards the mask is exactly what
+ * crisp_build_mask would have produced with keep_ratio = kkeep / nblk.  Typical use: build once with
+ * keep_ratio 1, let crisp_global_rank decide every layer's count, then reselect.
+ */
+CRISP_API crisp_status_t crisp_mask_reselect(crisp_mask_t mask, int32_t kkeep, const void *d_workspace,
+                                             void *stream);
+
+/* Algorithm 1's sparsity target kappa_p (fraction of ALL weights that are zero after step p) as the
+ * fraction of coarse blocks to prune when n of every m elements survive inside kept blocks:
+ * 1 - (1 - kappa) * m / n, clamped to [0, 1]. */
+CRISP_API crisp_status_t crisp_prune_fraction(double kappa, int32_t n, int32_t m, double *prune_fraction);
+
+/* The keep_ratio that makes crisp_keep_count return exactly kkeep for this layer. */
+CRISP_API crisp_status_t crisp_keep_ratio_for_count(const crisp_layer_desc_t *desc, int32_t kkeep,
+                                                    double *keep_ratio);
+
+/*
  * Same result as crisp_build_mask, for callers that cannot hand over a scratch workspace
  * because they are not allowed to allocate device memory at the point of the call (a plug-in
  * inside a framework that owns all device memory, a loop that must stay allocation-free after
@@ -190,6 +224,15 @@ CRISP_API crisp_status_t crisp_saliency_accumulate(const void *d_grad, int32_t g
 CRISP_API crisp_status_t crisp_saliency_finish(const float *d_acc, int64_t ld_acc, const uint16_t *d_w_bf16,
                                                int64_t ld_w, int32_t rows, int32_t k, int32_t samples,
                                                float *d_saliency, int64_t ld_s, void *stream);
+/* crisp_saliency_finish that also leaves the layer's largest score where crisp_build_mask_ex(...,
+ * CRISP_MASK_MAX_KNOWN) expects it: d_mask_workspace is that layer's mask workspace (crisp_mask_sizes; its
+ * first 256 bytes are cleared on `stream`, then the bits of max |S| - NaN read as 0, Inf as FLT_MAX - are
+ * written to its first word).  NULL makes this crisp_saliency_finish.  Eq. 1 / Algorithm 1: the score and the
+ * block scoring that follows it share one pass over the layer instead of two. */
+CRISP_API crisp_status_t crisp_saliency_finish_max(const float *d_acc, int64_t ld_acc, const uint16_t *d_w_bf16,
+                                                   int64_t ld_w, int32_t rows, int32_t k, int32_t samples,
+                                                   float *d_saliency, int64_t ld_s, void *d_mask_workspace,
+                                                   void *stream);
 
 /*
  * Global rank selection across the layers of a network: Algorithm 1 of the paper between the

@@ -247,3 +247,17 @@ def saliency(grads: np.ndarray, w_bits: np.ndarray) -> np.ndarray:
     if rc:
         raise ValueError(f"oracle_saliency rc={rc}")
     return out
+
+
+def saliency_f32(grads: np.ndarray, w_bits: np.ndarray) -> np.ndarray:
+    """Eq. 1 evaluated in fp32 in a fixed order (sum of the samples in order, times fp32(1/H), times W): the
+    evaluation to use where the score goes on to decide a mask that is compared bit for bit."""
+    g = np.ascontiguousarray(grads, dtype=np.float32)
+    w = np.ascontiguousarray(w_bits, dtype=np.uint16)
+    h, rows, k = g.shape
+    out = np.zeros((rows, k), dtype=np.float32)
+    rc = lib().oracle_saliency_f32(_p(g, C.c_float), C.c_int(h), _p(w, C.c_uint16), C.c_int(rows), C.c_int(k),
+                                   _p(out, C.c_float))
+    if rc:
+        raise ValueError(f"oracle_saliency_f32 rc={rc}")
+    return out

@@ -559,3 +559,25 @@ int oracle_saliency(const double *grads, int samples, const uint16_t *w, int row
     }
     return 0;
 }
+
+/*
+ * The same score in the precision and order in which a caller's fp32 accumulation produces it, for
+ * comparisons where the score decides integers downstream (the mask): the H gradients are added in the
+ * given order in fp32, the sum is multiplied by the fp32 reciprocal of H, then by the weight, each
+ * product rounded to fp32; out = |.|.  (Eq. 1 fixes neither precision nor order; this is one evaluation of
+ * it, within a few ulp of oracle_saliency.)  grads: H tensors [rows, k] as floats.
+ */
+int oracle_saliency_f32(const float *grads, int samples, const uint16_t *w, int rows, int k, float *out)
+{
+    if (!grads || !w || !out || samples <= 0 || rows <= 0 || k <= 0) return -1;
+    const int64_t n = (int64_t)rows * k;
+    const volatile float inv = 1.0f / (float)samples;
+    for (int64_t e = 0; e < n; ++e) {
+        volatile float sum = grads[e];
+        for (int i = 1; i < samples; ++i) sum = sum + grads[(int64_t)i * n + e];
+        volatile float t = sum * inv;              /* volatile: every step is rounded to fp32, nothing fused */
+        t = t * (float)bf16_to_double(w[e]);
+        out[e] = fabsf(t);
+    }
+    return 0;
+}

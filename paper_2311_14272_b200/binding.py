@@ -90,6 +90,11 @@ def load(path: Optional[str] = None):
         "crisp_spmm_conv": [vp, vp, P(ConvDesc), vp, i64, i32, vp],
         "crisp_saliency_accumulate": [vp, i32, i64, i32, i32, vp, i64, i32, vp],
         "crisp_saliency_finish": [vp, i64, vp, i64, i32, i32, i32, vp, i64, vp],
+        "crisp_saliency_finish_max": [vp, i64, vp, i64, i32, i32, i32, vp, i64, vp, vp],
+        "crisp_build_mask_ex": [vp, i64, P(LayerDesc), vp, vp, C.c_uint32, vp, P(vp)],
+        "crisp_mask_reselect": [vp, i32, vp, vp],
+        "crisp_prune_fraction": [C.c_double, i32, i32, P(C.c_double)],
+        "crisp_keep_ratio_for_count": [P(LayerDesc), i32, P(C.c_double)],
         "crisp_set_path": [vp, i32],
         "crisp_set_epilogue": [vp, vp, i32],
         "crisp_device_status": [vp, vp, P(i32)],
@@ -175,6 +180,38 @@ def crisp_saliency_finish(d_acc, ld_acc: int, d_w, ld_w: int, rows: int, k: int,
                           stream=None):
     _check(load().crisp_saliency_finish(_ptr(d_acc), ld_acc, _ptr(d_w), ld_w, rows, k, samples, _ptr(d_saliency), ld_s,
                                         _stream(stream)), "crisp_saliency_finish")
+
+
+def crisp_saliency_finish_max(d_acc, ld_acc: int, d_w, ld_w: int, rows: int, k: int, samples: int, d_saliency, ld_s: int,
+                              d_mask_workspace, stream=None):
+    _check(load().crisp_saliency_finish_max(_ptr(d_acc), ld_acc, _ptr(d_w), ld_w, rows, k, samples, _ptr(d_saliency),
+                                            ld_s, _ptr(d_mask_workspace), _stream(stream)), "crisp_saliency_finish_max")
+
+
+MASK_MAX_KNOWN = 1
+
+
+def crisp_build_mask_ex(d_saliency, ld_s: int, desc: LayerDesc, d_mask_buf, d_workspace, flags: int, stream=None) -> int:
+    out = C.c_void_p()
+    _check(load().crisp_build_mask_ex(_ptr(d_saliency), ld_s, C.byref(desc), _ptr(d_mask_buf), _ptr(d_workspace),
+                                      flags, _stream(stream), C.byref(out)), "crisp_build_mask_ex")
+    return out.value
+
+
+def crisp_mask_reselect(mask: int, kkeep: int, d_workspace, stream=None):
+    _check(load().crisp_mask_reselect(mask, kkeep, _ptr(d_workspace), _stream(stream)), "crisp_mask_reselect")
+
+
+def crisp_prune_fraction(kappa: float, n: int, m: int) -> float:
+    out = C.c_double()
+    _check(load().crisp_prune_fraction(float(kappa), n, m, C.byref(out)), "crisp_prune_fraction")
+    return out.value
+
+
+def crisp_keep_ratio_for_count(desc: LayerDesc, kkeep: int) -> float:
+    out = C.c_double()
+    _check(load().crisp_keep_ratio_for_count(C.byref(desc), kkeep, C.byref(out)), "crisp_keep_ratio_for_count")
+    return out.value
 
 
 def crisp_mask_scores(desc: LayerDesc, d_workspace):
@@ -354,12 +391,27 @@ class HybridLayer:
 
     def set_kkeep(self, kkeep: int):
         """Keep ratio that makes the next build_mask keep exactly `kkeep` blocks per row tile."""
-        self.desc.keep_ratio = float(kkeep) / float(self.nblk)
+        self.desc.keep_ratio = crisp_keep_ratio_for_count(self.desc, kkeep)
         self.nblk, self.kkeep = crisp_keep_count(self.desc)
         assert self.kkeep == kkeep
         mask_bytes, ws_bytes = crisp_mask_sizes(self.desc)
         if self.mask_buf.numel() < mask_bytes:
             self.mask_buf = self.torch.empty(mask_bytes, dtype=self.torch.uint8, device=self.device)
+        return self
+
+    def build_mask_max_known(self, saliency, stream=None):
+        """build_mask when the workspace already holds the layer maximum (crisp_saliency_finish_max wrote it)."""
+        assert saliency.is_cuda and saliency.dtype == self.torch.float32 and saliency.stride(1) == 1
+        crisp_mask_destroy(self.mask)
+        self.mask = crisp_build_mask_ex(saliency, saliency.stride(0), self.desc, self.mask_buf, self.workspace,
+                                        MASK_MAX_KNOWN, stream)
+        return self
+
+    def reselect(self, kkeep: int, stream=None):
+        """Keep only the `kkeep` best blocks per row tile of the mask just built (no pass over the saliency)."""
+        crisp_mask_reselect(self.mask, kkeep, self.workspace, stream)
+        self.desc.keep_ratio = crisp_keep_ratio_for_count(self.desc, kkeep)
+        self.kkeep = kkeep
         return self
 
     def export_mask(self, stream=None):
@@ -458,3 +510,59 @@ class HybridLayer:
             self.close()
         except Exception:
             pass
+
+
+class PruningNetwork:
+    """One pruning iteration of Algorithm 1 over all layers of a network, without the fine-tuning that follows it:
+
+        per layer   saliency of Eq. 1 from the caller's gradients   crisp_saliency_accumulate / _finish_max
+        per layer   N:M step and block scores (keep ratio 1)        crisp_build_mask_ex(MAX_KNOWN)
+        network     rank-column sums, global order, selection       crisp_global_rank
+        per layer   keep the selected number of blocks              crisp_mask_reselect
+        per layer   compress                                        crisp_encode
+
+    This class only owns buffers and issues those calls in that order; every number is computed by the library.
+    `shapes` is a list of (rows, k); the pattern (n:m, block shape) is shared by the layers.
+    """
+
+    def __init__(self, shapes, n, m, block_rows, block_k, min_keep=1, device="cuda"):
+        import torch
+        self.torch = torch
+        self.device = torch.device(device)
+        self.n, self.m = n, m
+        self.min_keep = min_keep
+        self.layers = [HybridLayer(r, k, n, m, block_rows, block_k, 1.0, device=device) for (r, k) in shapes]
+        self.acc = [torch.empty((r, k), dtype=torch.float32, device=self.device) for (r, k) in shapes]
+        self.sal = [torch.empty((r, k), dtype=torch.float32, device=self.device) for (r, k) in shapes]
+        self.rank_arr = make_rank_layers([L.rank_layer(min_keep) for L in self.layers])
+        self.rank_ws = torch.empty(crisp_global_rank_sizes(self.rank_arr), dtype=torch.uint8, device=self.device)
+        self.d_kkeep = torch.zeros(len(shapes), dtype=torch.int32, device=self.device)
+
+    def step(self, weights, grads, kappa, stream=None):
+        """weights[l]: bf16 CUDA tensor [rows, k]; grads[l]: list of H gradient tensors (bf16 or fp32) of that shape;
+        kappa: overall sparsity target of this iteration.  Returns the kept-block count of every layer; the layers'
+        masks and handles (self.layers[l]) hold the result."""
+        torch = self.torch
+        for L, w, gs, acc, s in zip(self.layers, weights, grads, self.acc, self.sal):
+            rows, k = L.desc.rows, L.desc.k
+            for i, g in enumerate(gs):
+                crisp_saliency_accumulate(g, 0 if g.dtype == torch.bfloat16 else 1, g.stride(0), rows, k, acc, k, i == 0,
+                                          stream)
+            crisp_saliency_finish_max(acc, k, w, w.stride(0), rows, k, len(gs), s, k, L.workspace, stream)
+            L.desc.keep_ratio = 1.0
+            L.nblk, L.kkeep = crisp_keep_count(L.desc)
+            L.build_mask_max_known(s, stream)
+        crisp_global_rank(self.rank_arr, crisp_prune_fraction(kappa, self.n, self.m), self.rank_ws, self.d_kkeep, stream)
+        if stream is None:
+            kk = self.d_kkeep.cpu().tolist()
+        else:
+            with torch.cuda.stream(stream):
+                kk = self.d_kkeep.cpu().tolist()
+        for L, w, c in zip(self.layers, weights, kk):
+            L.reselect(c, stream)
+            L.encode(w, stream)
+        return kk
+
+    def close(self):
+        for L in self.layers:
+            L.close()

@@ -103,7 +103,14 @@ crisp_status_t crisp_mask_sizes(const crisp_layer_desc_t *desc, size_t *mask_byt
 
 crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s, const crisp_layer_desc_t *desc,
                                 void *d_mask_buf, void *d_workspace, void *stream, crisp_mask_t *out) {
+    return crisp_build_mask_ex(d_saliency, ld_s, desc, d_mask_buf, d_workspace, 0, stream, out);
+}
+
+crisp_status_t crisp_build_mask_ex(const float *d_saliency, int64_t ld_s, const crisp_layer_desc_t *desc,
+                                   void *d_mask_buf, void *d_workspace, uint32_t flags, void *stream,
+                                   crisp_mask_t *out) {
     if (!out) return CRISP_INVALID_ARG;
+    if (flags & ~(uint32_t)CRISP_MASK_MAX_KNOWN) return CRISP_INVALID_ARG;
     *out = nullptr;
     Geometry g;
     crisp_status_t s = make_geometry(desc, &g);
@@ -119,9 +126,35 @@ crisp_status_t crisp_build_mask(const float *d_saliency, int64_t ld_s, const cri
     mk->d_nm_bits = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_mask_buf) + blk_col_bytes(g));
     mk->image_kind = image_kind(g);
     cudaError_t e = crisp::launch_build_mask(d_saliency, ld_s, g, mk->d_blk_col, mk->d_nm_bits, d_workspace,
-                                             crisp::mask_workspace_bytes(g), (cudaStream_t)stream);
+                                             crisp::mask_workspace_bytes(g), (flags & CRISP_MASK_MAX_KNOWN) != 0,
+                                             (cudaStream_t)stream);
     if (e != cudaSuccess) { delete mk; return CRISP_CUDA_ERROR; }
     *out = mk;
+    return CRISP_OK;
+}
+
+crisp_status_t crisp_mask_reselect(crisp_mask_t mask, int32_t kkeep, const void *d_workspace, void *stream) {
+    if (!mask || !d_workspace) return CRISP_INVALID_ARG;
+    if (kkeep < 0 || kkeep > mask->g.kkeep) return CRISP_INVALID_ARG;     // the kept sets are nested: only downwards
+    if (!aligned(d_workspace, kAlign)) return CRISP_INVALID_ARG;
+    mask->g.kkeep = kkeep;
+    cudaError_t e = crisp::launch_block_select(mask->g, d_workspace, mask->d_blk_col, mask->d_nm_bits, (cudaStream_t)stream);
+    return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
+}
+
+crisp_status_t crisp_prune_fraction(double kappa, int32_t n, int32_t m, double *prune_fraction) {
+    if (!prune_fraction || n < 1 || m < n || !(kappa >= 0.0) || kappa > 1.0) return CRISP_INVALID_ARG;
+    const double f = 1.0 - (1.0 - kappa) * (double)m / (double)n;
+    *prune_fraction = f < 0.0 ? 0.0 : (f > 1.0 ? 1.0 : f);
+    return CRISP_OK;
+}
+
+crisp_status_t crisp_keep_ratio_for_count(const crisp_layer_desc_t *desc, int32_t kkeep, double *keep_ratio) {
+    Geometry g;
+    crisp_status_t s = make_geometry(desc, &g);
+    if (s != CRISP_OK) return s;
+    if (!keep_ratio || kkeep < 0 || kkeep > g.nblk) return CRISP_INVALID_ARG;
+    *keep_ratio = (double)kkeep / (double)g.nblk;     // floor(ratio * nblk + 0.5) gives kkeep back
     return CRISP_OK;
 }
 

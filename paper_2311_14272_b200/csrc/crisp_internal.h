@@ -77,8 +77,11 @@ struct WalkArgs;
 
 // mask_kernels.cu
 cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, int32_t *d_blk_col,
-                              uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes,
+                              uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes, bool max_known,
                               cudaStream_t st);
+// per-row-tile selection alone, on the scores and group bits an earlier launch_build_mask left behind
+cudaError_t launch_block_select(const Geometry &g, const void *d_workspace, int32_t *d_blk_col, uint32_t *d_nm_bits,
+                                cudaStream_t st);
 size_t mask_workspace_bytes(const Geometry &g);
 
 // encode_kernels.cu

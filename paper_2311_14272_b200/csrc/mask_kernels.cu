@@ -302,34 +302,47 @@ size_t mask_workspace_bytes(const Geometry &g) {
     return kAlign + align_up((size_t)g.nrt * g.nblk * sizeof(unsigned long long));
 }
 
+cudaError_t launch_block_select(const Geometry &g, const void *d_workspace, int32_t *d_blk_col, uint32_t *d_nm_bits,
+                                cudaStream_t st) {
+    const unsigned long long *score =
+        reinterpret_cast<const unsigned long long *>(reinterpret_cast<const uint8_t *>(d_workspace) + kAlign);
+    const size_t smem = (size_t)g.nblk * (sizeof(unsigned long long) + sizeof(int));
+    if (smem + 64 > 48 * 1024) {     // the longest rows (nblk near 4096) need the opt-in shared-memory size
+        cudaError_t e = cudaFuncSetAttribute(block_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    block_select_kernel<<<dim3((unsigned)g.nrt, (unsigned)(g.bm / 32)), 256, smem, st>>>(g, score, d_blk_col, d_nm_bits);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, int32_t *d_blk_col,
-                              uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes,
+                              uint32_t *d_nm_bits, void *d_workspace, size_t workspace_bytes, bool max_known,
                               cudaStream_t st) {
     uint32_t *max_key = reinterpret_cast<uint32_t *>(d_workspace);
     unsigned long long *score =
         reinterpret_cast<unsigned long long *>(reinterpret_cast<uint8_t *>(d_workspace) + kAlign);
-    cudaError_t e = cudaMemsetAsync(d_workspace, 0, workspace_bytes, st);
+    // max_known: the first word already holds the layer's largest canonical |s| (written by the saliency kernel
+    // that produced S), so only the scores are cleared and the pass over S that finds the maximum is skipped
+    cudaError_t e = max_known ? cudaMemsetAsync(score, 0, workspace_bytes - kAlign, st)
+                              : cudaMemsetAsync(d_workspace, 0, workspace_bytes, st);
     if (e != cudaSuccess) return e;
     const bool vec_ok = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_s) & 15u) == 0);
 
-    const int64_t items = (int64_t)g.rows * ((g.k + 1023) / 1024);     // one warp per item
-    int grid0 = (int)((items + 7) / 8 < 148 * 8 ? (items + 7) / 8 : 148 * 8);
-    if (grid0 < 1) grid0 = 1;
-    max_key_kernel<<<grid0, 256, 0, st>>>(d_s, ld, g.rows, g.k, vec_ok, max_key);
+    if (!max_known) {
+        const int64_t items = (int64_t)g.rows * ((g.k + 1023) / 1024);     // one warp per item
+        int grid0 = (int)((items + 7) / 8 < 148 * 8 ? (items + 7) / 8 : 148 * 8);
+        if (grid0 < 1) grid0 = 1;
+        max_key_kernel<<<grid0, 256, 0, st>>>(d_s, ld, g.rows, g.k, vec_ok, max_key);
+    }
 
     dim3 grid1((unsigned)(g.mp() / kM1Rows), (unsigned)((g.kp() + kM1ChunkK - 1) / kM1ChunkK));
     if (g.m == 4)
         group_select_kernel<4><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
     else
         group_select_kernel<8><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
-
-    const size_t smem = (size_t)g.nblk * (sizeof(unsigned long long) + sizeof(int));
-    if (smem + 64 > 48 * 1024) {     // the longest rows (nblk near 4096) need the opt-in shared-memory size
-        e = cudaFuncSetAttribute(block_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    block_select_kernel<<<dim3((unsigned)g.nrt, (unsigned)(g.bm / 32)), 256, smem, st>>>(g, score, d_blk_col, d_nm_bits);
-    return cudaGetLastError();
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_block_select(g, d_workspace, d_blk_col, d_nm_bits, st);
 }
 
 }  // namespace crisp

@@ -48,12 +48,21 @@ saliency_accumulate_kernel(const void *__restrict__ grad, int64_t ld_g, int rows
     }
 }
 
+// |s| as the mask projection reads it (NaN -> 0, Inf -> FLT_MAX), as ordered bits
+__device__ __forceinline__ uint32_t canonical_key_bits(float v) {
+    return __float_as_uint(fminf(fmaxf(v, 0.f), 3.402823466e+38f));
+}
+
+// max_key != nullptr: the layer-wide maximum of the canonical score is left there as well (one atomic per warp),
+// which is the first thing the mask projection needs: it then does not have to stream S once more to find it.
 template <bool kVec>
 __global__ void __launch_bounds__(kSalThreads)
 saliency_finish_kernel(const float *__restrict__ acc, int64_t ld_a, const uint16_t *__restrict__ w, int64_t ld_w,
-                       int rows, int k, float inv_samples, float *__restrict__ s, int64_t ld_s) {
+                       int rows, int k, float inv_samples, float *__restrict__ s, int64_t ld_s,
+                       uint32_t *__restrict__ max_key) {
     const int kq = kVec ? k / 4 : k;
     const int64_t total = (int64_t)rows * kq;
+    uint32_t best = 0u;
     for (int64_t i = (int64_t)blockIdx.x * kSalThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kSalThreads) {
         const int r = (int)(i / kq), c = (int)(i - (int64_t)r * kq);
         if constexpr (kVec) {
@@ -65,20 +74,24 @@ saliency_finish_kernel(const float *__restrict__ acc, int64_t ld_a, const uint16
             o.z = fabsf(a.z * inv_samples * bf16_bits_to_float(raw.y & 0xFFFFu));
             o.w = fabsf(a.w * inv_samples * bf16_bits_to_float(raw.y >> 16));
             *reinterpret_cast<float4 *>(s + r * ld_s + 4 * c) = o;
+            best = max(max(best, canonical_key_bits(o.x)), max(canonical_key_bits(o.y), max(canonical_key_bits(o.z), canonical_key_bits(o.w))));
         } else {
-            s[r * ld_s + c] = fabsf(acc[r * ld_a + c] * inv_samples * bf16_bits_to_float(w[r * ld_w + c]));
+            const float v = fabsf(acc[r * ld_a + c] * inv_samples * bf16_bits_to_float(w[r * ld_w + c]));
+            s[r * ld_s + c] = v;
+            best = max(best, canonical_key_bits(v));
         }
+    }
+    if (max_key != nullptr) {
+        best = __reduce_max_sync(0xFFFFFFFFu, best);
+        if ((threadIdx.x & 31) == 0 && best) atomicMax(max_key, best);
     }
 }
 
 int wave_grid(int64_t work_items) {
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (sm_count <= 0) sm_count = 148;
-    }
+    int dev = 0, sm_count = 0;                               // asked for at every call: the current device may change
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+        sm_count = 148;
     const int64_t blocks = (work_items + kSalThreads - 1) / kSalThreads;
     const int64_t cap = (int64_t)sm_count * 8;               // 8 resident CTAs of 256 threads per SM
     return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
@@ -116,7 +129,14 @@ CRISP_API crisp_status_t crisp_saliency_accumulate(const void *d_grad, int32_t g
 CRISP_API crisp_status_t crisp_saliency_finish(const float *d_acc, int64_t ld_acc, const uint16_t *d_w_bf16, int64_t ld_w,
                                                int32_t rows, int32_t k, int32_t samples, float *d_saliency, int64_t ld_s,
                                                void *stream) {
+    return crisp_saliency_finish_max(d_acc, ld_acc, d_w_bf16, ld_w, rows, k, samples, d_saliency, ld_s, nullptr, stream);
+}
+
+CRISP_API crisp_status_t crisp_saliency_finish_max(const float *d_acc, int64_t ld_acc, const uint16_t *d_w_bf16,
+                                                   int64_t ld_w, int32_t rows, int32_t k, int32_t samples,
+                                                   float *d_saliency, int64_t ld_s, void *d_mask_workspace, void *stream) {
     using namespace crisp;
+    if (d_mask_workspace && reinterpret_cast<uintptr_t>(d_mask_workspace) % kAlign) return CRISP_INVALID_ARG;
     if (!d_acc || !d_w_bf16 || !d_saliency || samples <= 0) return CRISP_INVALID_ARG;
     if (rows <= 0 || k <= 0 || ld_acc < k || ld_w < k || ld_s < k) return CRISP_BAD_SHAPE;
     if (reinterpret_cast<uintptr_t>(d_acc) % 4 || reinterpret_cast<uintptr_t>(d_w_bf16) % 2 ||
@@ -126,8 +146,10 @@ CRISP_API crisp_status_t crisp_saliency_finish(const float *d_acc, int64_t ld_ac
     const int grid = wave_grid((int64_t)rows * (vec ? k / 4 : k));
     const float inv = 1.0f / (float)samples;
     cudaStream_t st = (cudaStream_t)stream;
-    if (vec) saliency_finish_kernel<true><<<grid, kSalThreads, 0, st>>>(d_acc, ld_acc, d_w_bf16, ld_w, rows, k, inv, d_saliency, ld_s);
-    else saliency_finish_kernel<false><<<grid, kSalThreads, 0, st>>>(d_acc, ld_acc, d_w_bf16, ld_w, rows, k, inv, d_saliency, ld_s);
+    uint32_t *max_key = reinterpret_cast<uint32_t *>(d_mask_workspace);
+    if (max_key && cudaMemsetAsync(max_key, 0, kAlign, st) != cudaSuccess) return CRISP_CUDA_ERROR;
+    if (vec) saliency_finish_kernel<true><<<grid, kSalThreads, 0, st>>>(d_acc, ld_acc, d_w_bf16, ld_w, rows, k, inv, d_saliency, ld_s, max_key);
+    else saliency_finish_kernel<false><<<grid, kSalThreads, 0, st>>>(d_acc, ld_acc, d_w_bf16, ld_w, rows, k, inv, d_saliency, ld_s, max_key);
     return cudaGetLastError() == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
 }
 

@@ -93,3 +93,21 @@ def test_saliency_score_hand_values_and_numpy():
     g2 = np.array([[[0.01, 0.01, 1.0, 1.0]]])
     s = oracle.saliency(g2, w2)[0]
     assert s[0] < s[1] and s[0] < s[2] and s[1] < s[3] and s[2] < s[3]
+
+
+def test_saliency_in_fp32_order_is_the_fp32_evaluation_and_close_to_fp64():
+    """oracle.saliency_f32: sum of the samples in order in fp32, times fp32(1/H), times W, each step rounded to fp32
+    (written out here with numpy's float32 scalars' arithmetic), and within a few ulp of the fp64 evaluation."""
+    rng = np.random.default_rng(4)
+    for h in (1, 3, 7):
+        g = (rng.standard_normal((h, 9, 20)) * 1e-2).astype(np.float32)
+        w = wl.f32_to_bf16_bits(rng.standard_normal((9, 20)).astype(np.float32))
+        acc = g[0].copy()
+        for i in range(1, h):
+            acc = (acc + g[i]).astype(np.float32)
+        inv = np.float32(1.0) / np.float32(h)
+        want = np.abs(((acc * inv).astype(np.float32) * wl.bf16_bits_to_f32(w)).astype(np.float32))
+        got = oracle.saliency_f32(g, w)
+        assert got.dtype == np.float32 and np.array_equal(got, want)
+        ref = oracle.saliency(g, w)
+        assert np.all(np.abs(got - ref) <= 4 * 2.0 ** -24 * (h + 2) * np.abs(g).mean(axis=0) * np.abs(wl.bf16_bits_to_f32(w)) + 1e-45)
