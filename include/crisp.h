@@ -347,19 +347,24 @@ CRISP_API crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, 
  *                                 * A[b, y + i - pad, x + j - pad, r]        (stride 1)
  *
  *   d_act_nhwc  [batch, height, width, channels] bf16, dense, 16-byte aligned
- *   d_y         [rows, batch*ho*wo] bf16 (y_dtype 0) or fp32 (1), leading dimension ldy,
+ *   d_y         y_layout 0: [rows, batch*ho*wo] bf16 (y_dtype 0) or fp32 (1), leading dimension ldy >=
+ *               batch*ho*wo; y_layout 1: [batch, ho, wo, ldy] (NHWC, output channel fastest, ldy >= rows
+ *               elements between pixels), which is the d_act_nhwc of the next convolution as it stands,
+ *               so that layers chain without a transposition;
  *               ho = height + 2*pad - kernel_h + 1, wo likewise
  * The handle's k must equal kernel_h*kernel_w*channels (BAD_SHAPE otherwise).  Supported
  * (UNSUPPORTED otherwise; lower the convolution to a matrix and call crisp_spmm): block_k = 64,
  * channels a multiple of 64, a tensor-core execution image and at least one kept block.  Y is
  * written by bulk tensor stores when d_y is 16-byte aligned and wo*sizeof(Y element) and
- * ldy*sizeof(Y element) are multiples of 16 bytes, element by element otherwise (e.g. 28- or
- * 14-pixel rows of bf16).  Same tolerance and status reporting as crisp_spmm.
+ * ldy*sizeof(Y element) are multiples of 16 bytes (NHWC: when ldy*sizeof(Y element) is), element by
+ * element otherwise (e.g. 28- or 14-pixel rows of bf16).  Same tolerance and status reporting as
+ * crisp_spmm.
  */
 typedef struct {
     int32_t batch, height, width, channels;   /* input activation, NHWC                         */
     int32_t kernel_h, kernel_w;               /* filter taps                                    */
     int32_t pad;                              /* zero padding on every side                     */
+    int32_t y_layout;                         /* 0: Y [rows, batch*ho*wo]; 1: Y NHWC [batch, ho, wo, ldy] */
 } crisp_conv_desc_t;
 
 CRISP_API crisp_status_t crisp_spmm_conv(crisp_handle_t handle, const uint16_t *d_act_nhwc,

@@ -31,7 +31,7 @@ class RankLayer(C.Structure):
 
 class ConvDesc(C.Structure):
     _fields_ = [("batch", C.c_int32), ("height", C.c_int32), ("width", C.c_int32), ("channels", C.c_int32),
-                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad", C.c_int32)]
+                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad", C.c_int32), ("y_layout", C.c_int32)]
 
 
 class LaunchInfo(C.Structure):
@@ -459,16 +459,19 @@ class HybridLayer:
         crisp_spmm(self.handle, x, x.stride(0), ncols, y, y.stride(0), y_dtype, stream)
         return y
 
-    def spmm_conv(self, act_nhwc, kernel_h, kernel_w, pad, y=None, y_dtype=0, stream=None):
-        """Convolution (stride 1) of an NHWC bf16 activation with this layer's weights, without an X matrix."""
+    def spmm_conv(self, act_nhwc, kernel_h, kernel_w, pad, y=None, y_dtype=0, stream=None, nhwc_out=False):
+        """Convolution (stride 1) of an NHWC bf16 activation with this layer's weights, without an X matrix.
+        nhwc_out: Y is [batch, ho, wo, rows] (the next convolution's activation) instead of [rows, batch*ho*wo]."""
         torch = self.torch
         assert act_nhwc.is_cuda and act_nhwc.element_size() == 2 and act_nhwc.is_contiguous() and act_nhwc.dim() == 4
         b, h, w, c = act_nhwc.shape
         ho, wo = h + 2 * pad - kernel_h + 1, w + 2 * pad - kernel_w + 1
+        dt = torch.float32 if y_dtype else torch.bfloat16
         if y is None:
-            y = torch.empty((self.desc.rows, b * ho * wo), dtype=torch.float32 if y_dtype else torch.bfloat16,
+            y = torch.empty((b, ho, wo, self.desc.rows) if nhwc_out else (self.desc.rows, b * ho * wo), dtype=dt,
                             device=self.device)
-        crisp_spmm_conv(self.handle, act_nhwc, ConvDesc(b, h, w, c, kernel_h, kernel_w, pad), y, y.stride(0),
+        ldy = y.stride(2) if nhwc_out else y.stride(0)
+        crisp_spmm_conv(self.handle, act_nhwc, ConvDesc(b, h, w, c, kernel_h, kernel_w, pad, 1 if nhwc_out else 0), y, ldy,
                         y_dtype, stream)
         return y
 

@@ -314,12 +314,14 @@ crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, con
     if (cd->batch <= 0 || cd->height <= 0 || cd->width <= 0 || cd->channels <= 0 || cd->kernel_h <= 0 ||
         cd->kernel_w <= 0 || cd->pad < 0)
         return CRISP_BAD_SHAPE;
+    if (cd->y_layout != 0 && cd->y_layout != 1) return CRISP_INVALID_ARG;
     crisp::ConvGeom cg{cd->batch, cd->height, cd->width, cd->channels, cd->kernel_h, cd->kernel_w, cd->pad,
-                       cd->height + 2 * cd->pad - cd->kernel_h + 1, cd->width + 2 * cd->pad - cd->kernel_w + 1};
+                       cd->height + 2 * cd->pad - cd->kernel_h + 1, cd->width + 2 * cd->pad - cd->kernel_w + 1,
+                       cd->y_layout};
     if (cg.ho <= 0 || cg.wo <= 0) return CRISP_BAD_SHAPE;
     if ((int64_t)cd->kernel_h * cd->kernel_w * cd->channels != h->g.k) return CRISP_BAD_SHAPE;
     const int64_t ncols = (int64_t)cg.batch * cg.ho * cg.wo;
-    if (ldy < ncols) return CRISP_BAD_SHAPE;
+    if (ldy < (cg.nhwc_out ? (int64_t)h->g.rows : ncols)) return CRISP_BAD_SHAPE;
     const int es = y_dtype ? 4 : 2;
     // the gather needs whole k-blocks inside one filter tap, 128-byte channel slabs, and TMA-addressable tensors
     if (h->g.bk != 64 || cd->channels % h->g.bk != 0) return CRISP_UNSUPPORTED;

@@ -113,7 +113,7 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
                                cudaStream_t st);
 bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols);
 // Convolution geometry for the implicit-GEMM mode (stride 1): NHWC activation, ho x wo output pixels.
-struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo; };
+struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo, nhwc_out; };
 // conv == nullptr: d_x is the [k, ncols] matrix.  Otherwise d_x is the activation and ncols = batch*ho*wo.
 // `h->plan` is reused when the operands, shape and epilogue are those of the previous call; `h->last` is filled in.
 cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols,

@@ -1,13 +1,13 @@
 // Mask projection kernels: saliency -> hybrid (block + N:M) mask.
 //
 // Algorithm 1 of the paper, restricted to one layer with the block keep count given:
-//   K-M0  layer-wide maximum of the canonical saliency (sets the fixed-point scale)
-//   K-M1  per group of M: keep the N largest (fine-grained N:M step) and accumulate the
-//         block scores s_j = sum |T_w| as exact fixed-point integers
+//   K-M1a per group of M: keep the N largest (fine-grained N:M step), and the layer-wide maximum
+//         of the canonical saliency (it sets the fixed-point scale): one pass over S from HBM
+//   K-M1b block scores s_j = sum |T_w| as exact fixed-point integers: second pass over S, which
+//         for layers up to the size of L2 is served from there
 //   K-M2  per row of the block grid: keep the kkeep highest-scored blocks and clear the
 //         bits of the pruned ones (blocks keep their positions)
-// All three stream the data once with coalesced 32-byte-per-lane accesses; the work is
-// bound by HBM bandwidth (one compare network per 4 bytes read).
+// Coalesced 32-byte-per-lane accesses; K-M1a is bound by HBM bandwidth.
 #include "crisp_internal.h"
 
 namespace crisp {
@@ -60,46 +60,6 @@ __device__ __forceinline__ void load8(const float *__restrict__ s, int64_t ld, i
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) key[i] = (k0 + i < k) ? canonical_key(__ldg(p + i)) : 0u;
-    }
-}
-
-// K-M0.  One warp per (row, 1024-element segment): eight 16-byte loads per lane are issued before
-// any is used, partial maxima are combined per warp and per CTA, one atomic per CTA.
-__global__ void __launch_bounds__(256)
-max_key_kernel(const float *__restrict__ s, int64_t ld, int rows, int k, bool vec_ok,
-               uint32_t *__restrict__ max_key) {
-    __shared__ uint32_t s_best[8];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int segs = (k + 1023) / 1024;
-    const int64_t items = (int64_t)rows * segs;
-    const int64_t nwarps = (int64_t)gridDim.x * 8;
-    uint32_t best = 0u;
-    for (int64_t it = (int64_t)blockIdx.x * 8 + warp; it < items; it += nwarps) {
-        const int64_t row = it / segs;
-        const int64_t k0 = (it - row * segs) * 1024 + lane * 8;
-        uint32_t key[4][8];
-        if (vec_ok && (it - row * segs) * 1024 + 1024 <= k) {       // whole segment inside the row
-#pragma unroll
-            for (int pass = 0; pass < 4; ++pass) load8_raw(s, ld, row, k0 + pass * 256, key[pass]);
-#pragma unroll
-            for (int pass = 0; pass < 4; ++pass)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) best = max(best, canonical_bits(key[pass][j]));
-        } else {
-#pragma unroll
-            for (int pass = 0; pass < 4; ++pass) load8(s, ld, rows, k, row, k0 + pass * 256, vec_ok, key[pass]);
-#pragma unroll
-            for (int pass = 0; pass < 4; ++pass)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) best = max(best, key[pass][j]);
-        }
-    }
-    best = __reduce_max_sync(0xFFFFFFFFu, best);
-    if (lane == 0) s_best[warp] = best;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < 8; ++w) best = max(best, s_best[w]);
-        if (best) atomicMax(max_key, best);
     }
 }
 
@@ -161,42 +121,27 @@ __device__ __forceinline__ uint32_t keep_mask_of_outcomes(uint32_t o, int n) {
     return (uint32_t)(r0 < n) | ((uint32_t)(r1 < n) << 1) | ((uint32_t)(r2 < n) << 2) | ((uint32_t)(r3 < n) << 3);
 }
 
-constexpr int kM1Rows = 32;              // rows per CTA of K-M1 (divides every block height)
+constexpr int kM1Rows = 32;              // rows per work item of K-M1a / K-M1b (divides every block height)
 constexpr int kM1RowsPerWarp = kM1Rows / (kM1Threads / 32);
 
-// K-M1.  One CTA covers 32 rows x 256 k-elements.  Warp w takes rows 4w..4w+3 (all loads issued
-// first); lane l owns the 8 elements at k = chunk*256 + 8*l of each row, so a lane stays inside one
-// block column and keeps its partial block score in a register.  A lane stores its eight mask bits as
-// one byte; four lanes add up one partial score (a word never straddles a block: block_k is a multiple of 32).
-template <int M>
-__global__ void __launch_bounds__(kM1Threads)
-group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_ok,
-                    const uint32_t *__restrict__ max_key, uint32_t *__restrict__ nm_bits,
-                    unsigned long long *__restrict__ score) {
-    __shared__ unsigned long long s_score[kM1ChunkK / 32 + 2];
-    __shared__ uint8_t s_keep[64];
-    if (M == 4 && threadIdx.x < 64) s_keep[threadIdx.x] = (uint8_t)keep_mask_of_outcomes(threadIdx.x, g.n);
-    const int chunk = blockIdx.y;
-    const int64_t row0 = (int64_t)blockIdx.x * kM1Rows;
-    const int rt = (int)(row0 / g.bm);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t k0 = (int64_t)chunk * kM1ChunkK + lane * 8;
-    const int first_blk = (chunk * kM1ChunkK) / g.bk;
-    if (threadIdx.x < kM1ChunkK / 32 + 2) s_score[threadIdx.x] = 0ull;
-    __syncthreads();
+// One work item = 32 rows x 256 k-elements.  Warp w takes rows 4w..4w+3 (all loads issued first); lane l owns
+// the 8 elements at k = chunk*256 + 8*l of each row, so a lane stays inside one block column.  Items are dealt
+// out to a grid of resident CTAs (grid-stride), chunk fastest, so that a CTA streams along rows.
+struct M1Item { int64_t row0; int chunk; };
+__device__ __forceinline__ M1Item m1_item(int64_t it, int chunks) {
+    M1Item x;
+    const int64_t rg = it / chunks;
+    x.chunk = (int)(it - rg * chunks);
+    x.row0 = rg * kM1Rows;
+    return x;
+}
 
-    const uint32_t mk = *max_key;
-    const int e_max = mk ? key_exponent(mk) : 0;
-    // floor(value * 2^(40 - e_max)): when that power of two is an fp32 number, the product is exact
-    // (value <= layer maximum, so it stays below 2^41) and one round-down conversion gives the floor
-    const int scale_exp = kScoreFractionBits - e_max;
-    const bool float_scale = scale_exp >= -126 && scale_exp <= 127;
-    const float scale = float_scale ? __uint_as_float((uint32_t)(127 + scale_exp) << 23) : 0.f;
-    const bool in_kp = k0 < g.kp();
-    uint32_t key[kM1RowsPerWarp][8];
-    if (vec_ok && row0 + kM1Rows <= g.rows && (int64_t)(chunk + 1) * kM1ChunkK <= g.k) {   // interior tile
+// The 8 canonical keys of the lane's elements of row `row` (zero beyond the matrix).
+__device__ __forceinline__ void m1_load_rows(const float *__restrict__ s, int64_t ld, const Geometry &g, bool vec_ok,
+                                             const M1Item &x, int warp, int64_t k0, uint32_t key[kM1RowsPerWarp][8]) {
+    if (vec_ok && x.row0 + kM1Rows <= g.rows && (int64_t)(x.chunk + 1) * kM1ChunkK <= g.k) {   // interior item
 #pragma unroll
-        for (int i = 0; i < kM1RowsPerWarp; ++i) load8_raw(s, ld, row0 + warp * kM1RowsPerWarp + i, k0, key[i]);
+        for (int i = 0; i < kM1RowsPerWarp; ++i) load8_raw(s, ld, x.row0 + warp * kM1RowsPerWarp + i, k0, key[i]);
 #pragma unroll
         for (int i = 0; i < kM1RowsPerWarp; ++i)
 #pragma unroll
@@ -204,39 +149,133 @@ group_select_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool ve
     } else {
 #pragma unroll
         for (int i = 0; i < kM1RowsPerWarp; ++i)
-            load8(s, ld, g.rows, g.k, row0 + warp * kM1RowsPerWarp + i, k0, vec_ok, key[i]);
+            load8(s, ld, g.rows, g.k, x.row0 + warp * kM1RowsPerWarp + i, k0, vec_ok, key[i]);
     }
-    unsigned long long acc = 0ull;
-#pragma unroll
-    for (int i = 0; i < kM1RowsPerWarp; ++i) {
-        const int64_t row = row0 + warp * kM1RowsPerWarp + i;
-        uint32_t bits;
-        if constexpr (M == 4)
-            bits = (uint32_t)s_keep[outcomes4(key[i])] | ((uint32_t)s_keep[outcomes4(key[i] + 4)] << 4);
-        else
-            bits = top_n_bits<M>(key[i], g.n);
-        const uint32_t counted = g.score_mode == 0 ? bits : 0xFFu;
-        if (float_scale) {                   // uniform over the grid; all-zero layers give scale * 0 = 0
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if ((counted >> j) & 1u) acc += __float2ull_rd(__uint_as_float(key[i][j]) * scale);
-        } else if (mk) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if ((counted >> j) & 1u) acc += fixed_point_score(key[i][j], e_max);
-        }
-        // the lane's eight bits are byte (k0 / 8) mod 4 of their little-endian mask word: a warp stores 32
-        // consecutive bytes of the row
-        if (in_kp) reinterpret_cast<uint8_t *>(nm_bits + row * g.wpr)[k0 >> 3] = (uint8_t)bits;
-    }
-    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
-    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
-    if ((lane & 3) == 0 && in_kp && acc) atomicAdd(&s_score[(int)(k0 / g.bk) - first_blk], acc);
+}
+
+// K-M1a: the fine-grained N:M step (which does not depend on the score scale) and the layer maximum (which fixes
+// the scale) in ONE pass over S, the pass that comes from HBM: per group of M the N largest are marked, a lane
+// stores its eight mask bits as one byte, and the largest key goes to max_key (one atomic per CTA).
+// find_max = false when the caller already knows the maximum.
+template <int M>
+__global__ void __launch_bounds__(kM1Threads)
+group_bits_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_ok, int64_t items, int chunks,
+                  bool find_max, uint32_t *__restrict__ max_key, uint32_t *__restrict__ nm_bits) {
+    __shared__ uint8_t s_keep[64];
+    __shared__ uint32_t s_best[kM1Threads / 32];
+    if (M == 4 && threadIdx.x < 64) s_keep[threadIdx.x] = (uint8_t)keep_mask_of_outcomes(threadIdx.x, g.n);
     __syncthreads();
-    if (threadIdx.x < kM1ChunkK / 32 + 2) {
-        const int jb = first_blk + threadIdx.x;
-        const unsigned long long v = s_score[threadIdx.x];
-        if (jb < g.nblk && v) atomicAdd(&score[(int64_t)rt * g.nblk + jb], v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t best = 0u;
+    for (int64_t it = blockIdx.x; it < items; it += gridDim.x) {
+        const M1Item x = m1_item(it, chunks);
+        const int64_t k0 = (int64_t)x.chunk * kM1ChunkK + lane * 8;
+        uint32_t key[kM1RowsPerWarp][8];
+        m1_load_rows(s, ld, g, vec_ok, x, warp, k0, key);
+        const bool in_kp = k0 < g.kp();
+#pragma unroll
+        for (int i = 0; i < kM1RowsPerWarp; ++i) {
+            const int64_t row = x.row0 + warp * kM1RowsPerWarp + i;
+            uint32_t bits;
+            if constexpr (M == 4)
+                bits = (uint32_t)s_keep[outcomes4(key[i])] | ((uint32_t)s_keep[outcomes4(key[i] + 4)] << 4);
+            else
+                bits = top_n_bits<M>(key[i], g.n);
+            // the lane's eight bits are byte (k0 / 8) mod 4 of their little-endian mask word: a warp stores 32
+            // consecutive bytes of the row
+            if (in_kp) reinterpret_cast<uint8_t *>(nm_bits + row * g.wpr)[k0 >> 3] = (uint8_t)bits;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) best = max(best, key[i][j]);
+        }
+    }
+    if (find_max) {
+        best = __reduce_max_sync(0xFFFFFFFFu, best);
+        if (lane == 0) s_best[warp] = best;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int w = 1; w < kM1Threads / 32; ++w) best = max(best, s_best[w]);
+            if (best) atomicMax(max_key, best);
+        }
+    }
+}
+
+// floor(v) of an fp32 value 0 <= v < 2^41 without a float-to-integer conversion per element (those run at a
+// fraction of the fp32 rate and were what bound this kernel): v = r + d with r = v rounded to a multiple of 2^20
+// (adding and subtracting 1.5 * 2^43 does that, exactly) and d = v - r exact, |d| <= 2^19; floor(d) by the same
+// device with 1.5 * 2^23 and a correction where it rounded up.  r and floor(d) are then added up in fp32 over the
+// eight elements of a row, which is exact (r / 2^20 <= 2^21 each, |floor(d)| <= 2^19 each), and converted once.
+__device__ __forceinline__ void floor_parts(float v, float &r, float &fd) {
+    r = __fsub_rn(__fadd_rn(v, 13194139533312.f), 13194139533312.f);            // 1.5 * 2^43
+    const float d = __fsub_rn(v, r);
+    const float t = __fsub_rn(__fadd_rn(d, 12582912.f), 12582912.f);            // 1.5 * 2^23: d to the nearest integer
+    fd = t > d ? __fsub_rn(t, 1.f) : t;
+}
+
+// K-M1b: the block scores s_j = sum |T_w| as exact fixed-point integers, once the scale is known.  Second pass
+// over S (for layers that fit, out of L2, where K-M1a left it).  Warps are independent (no shared memory, no
+// barrier): a lane adds floor(|s| * 2^(40 - e_max)) of its counted elements (the N:M survivors, read back as the
+// byte K-M1a stored, or all of them) over its warp's four rows, the four lanes of a 32-element word add up
+// (a mask word never straddles a block: block_k is a multiple of 32), and one lane per word adds the partial
+// score to the block's 64-bit total with an atomic (integer addition: any order gives the same sum).
+__global__ void __launch_bounds__(kM1Threads)
+block_score_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_ok, int64_t items, int chunks,
+                   const uint32_t *__restrict__ max_key, const uint32_t *__restrict__ nm_bits,
+                   unsigned long long *__restrict__ score) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t mk = *max_key;
+    if (!mk) return;                                         // an all-zero layer: every score stays 0
+    const int e_max = key_exponent(mk);
+    // floor(value * 2^(40 - e_max)): when that power of two is an fp32 number, the product is exact
+    // (value <= layer maximum, so it stays below 2^41)
+    const int scale_exp = kScoreFractionBits - e_max;
+    const bool float_scale = scale_exp >= -126 && scale_exp <= 127;
+    const float scale = float_scale ? __uint_as_float((uint32_t)(127 + scale_exp) << 23) : 0.f;
+    for (int64_t it = blockIdx.x; it < items; it += gridDim.x) {
+        const M1Item x = m1_item(it, chunks);
+        const int64_t k0 = (int64_t)x.chunk * kM1ChunkK + lane * 8;
+        const int rt = (int)(x.row0 / g.bm);
+        uint32_t key[kM1RowsPerWarp][8];
+        m1_load_rows(s, ld, g, vec_ok, x, warp, k0, key);
+        const bool in_kp = k0 < g.kp();
+        unsigned long long acc = 0ull;
+        if (float_scale) {
+#pragma unroll
+            for (int i = 0; i < kM1RowsPerWarp; ++i) {
+                const int64_t row = x.row0 + warp * kM1RowsPerWarp + i;
+                uint32_t counted = 0xFFu;
+                if (g.score_mode == 0) counted = in_kp ? reinterpret_cast<const uint8_t *>(nm_bits + row * g.wpr)[k0 >> 3] : 0u;
+                float r_sum = 0.f, d_sum = 0.f;              // exact: see floor_parts
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float r, fd;
+                    floor_parts(__uint_as_float(key[i][j]) * scale, r, fd);
+                    if ((counted >> j) & 1u) { r_sum = __fadd_rn(r_sum, r); d_sum = __fadd_rn(d_sum, fd); }
+                }
+                acc += ((unsigned long long)__float2uint_rn(r_sum * 9.5367431640625e-07f) << 20) + (long long)__float2int_rn(d_sum);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < kM1RowsPerWarp; ++i) {
+                const int64_t row = x.row0 + warp * kM1RowsPerWarp + i;
+                uint32_t counted = 0xFFu;
+                if (g.score_mode == 0) counted = in_kp ? reinterpret_cast<const uint8_t *>(nm_bits + row * g.wpr)[k0 >> 3] : 0u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if ((counted >> j) & 1u) acc += fixed_point_score(key[i][j], e_max);
+            }
+        }
+        acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
+        acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
+        // lanes that share a block column (block_k / 8 of them, 4, 8, 12 or 16): add up as far as the lane groups
+        // of a power of two allow, then one atomic per group
+        if (g.bk % 64 == 0) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 4);
+        if (g.bk % 128 == 0) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 8);
+        const int grp = g.bk % 128 == 0 ? 15 : (g.bk % 64 == 0 ? 7 : 3);
+        if ((lane & grp) == 0 && in_kp && acc) {
+            const int jb = (int)(k0 / g.bk);
+            if (jb < g.nblk) atomicAdd(&score[(int64_t)rt * g.nblk + jb], acc);
+        }
     }
 }
 
@@ -328,18 +367,28 @@ cudaError_t launch_build_mask(const float *d_s, int64_t ld, const Geometry &g, i
     if (e != cudaSuccess) return e;
     const bool vec_ok = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_s) & 15u) == 0);
 
-    if (!max_known) {
-        const int64_t items = (int64_t)g.rows * ((g.k + 1023) / 1024);     // one warp per item
-        int grid0 = (int)((items + 7) / 8 < 148 * 8 ? (items + 7) / 8 : 148 * 8);
-        if (grid0 < 1) grid0 = 1;
-        max_key_kernel<<<grid0, 256, 0, st>>>(d_s, ld, g.rows, g.k, vec_ok, max_key);
-    }
-
-    dim3 grid1((unsigned)(g.mp() / kM1Rows), (unsigned)((g.kp() + kM1ChunkK - 1) / kM1ChunkK));
+    // work items of 32 rows x 256 k-elements, dealt out to at most eight resident CTAs per SM
+    const int chunks = (int)((g.kp() + kM1ChunkK - 1) / kM1ChunkK);
+    const int64_t items = (g.mp() / kM1Rows) * chunks;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    // grids of resident CTAs: every CTA is on an SM from the start and takes its share of the items
+    auto resident_grid = [&](const void *kern) {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kM1Threads, 0) != cudaSuccess || per_sm <= 0) per_sm = 4;
+        const int64_t cap = (int64_t)sms * per_sm;
+        return (int)(items < cap ? items : cap);
+    };
     if (g.m == 4)
-        group_select_kernel<4><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
+        group_bits_kernel<4><<<resident_grid((const void *)group_bits_kernel<4>), kM1Threads, 0, st>>>(
+            d_s, ld, g, vec_ok, items, chunks, !max_known, max_key, d_nm_bits);
     else
-        group_select_kernel<8><<<grid1, kM1Threads, 0, st>>>(d_s, ld, g, vec_ok, max_key, d_nm_bits, score);
+        group_bits_kernel<8><<<resident_grid((const void *)group_bits_kernel<8>), kM1Threads, 0, st>>>(
+            d_s, ld, g, vec_ok, items, chunks, !max_known, max_key, d_nm_bits);
+    block_score_kernel<<<resident_grid((const void *)block_score_kernel), kM1Threads, 0, st>>>(
+        d_s, ld, g, vec_ok, items, chunks, max_key, d_nm_bits, score);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return launch_block_select(g, d_workspace, d_blk_col, d_nm_bits, st);

@@ -55,6 +55,7 @@ struct TcParams {
     int cv_plain;               // Y rows are not TMA-addressable (wo * element size not a multiple of 16 bytes):
                                 // the epilogue stores element by element
     int cv_tw_log2, cv_img_log2;   // log2(tw), log2(tw * th)
+    int cv_nhwc;                // Y is [batch, ho, wo, ldy] (output channel fastest): the next convolution's activation
     // Thin layers (one CTA tile, at most 128 / stack rows; matrix mode): a tile covers `stack` column tiles, one per
     // group of 128 / stack accumulator lanes.  For group q the walk is run again with the image copy whose weights
     // sit in that group's rows (all other rows zero) against the X columns of column tile ct * stack + q.
@@ -199,6 +200,54 @@ __device__ __forceinline__ void store_chunk(const TcParams &p, const CUtensorMap
         }
         slot = (slot + 1) & (p.stg_bufs - 1);
     }
+}
+
+// One epilogue chunk of a convolution whose output is NHWC: the lane holds one output channel (row y0 + lane) of
+// kOutCols pixels, memory wants the 32 channels of a pixel side by side.  The chunk is transposed through the
+// warp's staging tile, [pixel][32 channels] (64 or 128 bytes per pixel, 4096 bytes per chunk), and goes out
+// as one 4-D bulk tensor store of {32 channels, tw, pixels / tw, 1} (it clips channels beyond `rows` and pixels
+// outside the images), or, where the pixel pitch is not a multiple of 16 bytes, pixel by pixel with the 32
+// lanes on consecutive channels.  `out` is packed as in store_chunk (bf16: pixels 2i, 2i+1 in word i).
+template <typename OutT>
+__device__ __forceinline__ void store_chunk_nhwc(const TcParams &p, const CUtensorMap *map_y, uint32_t stg, uint8_t *stg_gen,
+                                                 int lane, const uint32_t (&out)[32], const TileOrigin &org, int col0, int y0) {
+    constexpr int kOutCols = 128 / (int)sizeof(OutT);
+    constexpr int kRowBytes = 32 * (int)sizeof(OutT);           // one pixel: 32 channels
+    const int per_image = p.cv_tw * p.cv_th;
+    const int img = col0 / per_image;
+    const int cx = org.x, cy = org.y + (col0 - img * per_image) / p.cv_tw, cb = org.b + img;
+    if (y0 >= p.rows) return;
+    if (lane == 0 && !p.cv_plain) bulk_wait_read<0>();          // the previous store has finished reading the tile
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        if constexpr (sizeof(OutT) == 2) {
+            *reinterpret_cast<uint16_t *>(stg_gen + (2 * i) * kRowBytes + lane * 2) = (uint16_t)(out[i] & 0xFFFFu);
+            *reinterpret_cast<uint16_t *>(stg_gen + (2 * i + 1) * kRowBytes + lane * 2) = (uint16_t)(out[i] >> 16);
+        } else {
+            *reinterpret_cast<uint32_t *>(stg_gen + i * kRowBytes + lane * 4) = out[i];
+        }
+    }
+    if (!p.cv_plain) {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            if (cx < p.cv_wo && cy < p.cv_ho && cb < p.cv_batch) tma_store_4d(map_y, stg, y0, cx, cy, cb);
+            bulk_commit();
+        }
+        return;
+    }
+    __syncwarp();
+    const bool row_ok = y0 + lane < p.rows;
+    for (int c = 0; c < kOutCols; ++c) {
+        const int col = col0 + c;
+        const int im = col >> p.cv_img_log2, rem = col & ((1 << p.cv_img_log2) - 1);
+        const int gy = org.y + (rem >> p.cv_tw_log2), gx = org.x + (rem & (p.cv_tw - 1)), gb = org.b + im;
+        if (row_ok && gx < p.cv_wo && gy < p.cv_ho && gb < p.cv_batch)
+            reinterpret_cast<OutT *>(p.y)[(((int64_t)gb * p.cv_ho + gy) * p.cv_wo + gx) * p.ldy + y0 + lane] =
+                *reinterpret_cast<const OutT *>(stg_gen + c * kRowBytes + lane * (int)sizeof(OutT));
+    }
+    __syncwarp();
 }
 
 // The MMA issuer's loop, with the number of MMAs per kept block (NM) fixed at compile time: the loop is
@@ -484,7 +533,8 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 32; ++i) out[i] = accr[c * 32 + i];
                     }
-                    store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, half * kWarpCols + c * kOutCols, y0, slot);
+                    if (kConv && p.cv_nhwc) store_chunk_nhwc<OutT>(p, &map_y, stg, stg_gen, lane, out, org, half * kWarpCols + c * kOutCols, y0);
+                    else store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, half * kWarpCols + c * kOutCols, y0, slot);
                 }
             } else {
                 if (half == 0) {
@@ -516,7 +566,8 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                                 for (int i = 0; i < 32; ++i) out[i] = __float_as_uint(fmaxf(__uint_as_float(out[i]) + bias_v, floor_v));
                             }
                         }
-                        store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0, slot);
+                        if (kConv && p.cv_nhwc) store_chunk_nhwc<OutT>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0);
+                        else store_chunk<OutT, kConv>(p, &map_y, stg, stg_gen, lane, out, org, c * kOutCols, y0, slot);
                     }
                 }
                 tc_fence_before();
@@ -782,11 +833,12 @@ bool make_map_image(CUtensorMap *map, const void *image, uint64_t total_bytes, u
 // inner box: 128, 64 or 32 bytes, none for 16.  (A store through a map whose span is wider than its inner
 // box raised an illegal memory access on B200, although the map encodes.)
 bool make_map_4d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, const uint64_t (&dims)[4],
-                 const uint64_t (&strides_bytes)[3], const uint32_t (&box)[4]) {
+                 const uint64_t (&strides_bytes)[3], const uint32_t (&box)[4], bool swizzle) {
     EncodeTiledFn fn = encode_tiled_fn();
     const uint64_t inner = (uint64_t)box[0] * elem_bytes;
     if (!fn || (inner != 128 && inner != 64 && inner != 32 && inner != 16)) return false;
-    const CUtensorMapSwizzle swz = inner == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+    const CUtensorMapSwizzle swz = !swizzle ? CU_TENSOR_MAP_SWIZZLE_NONE
+                                 : inner == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
                                  : inner == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
     cuuint64_t d[4] = {dims[0], dims[1], dims[2], dims[3]};
     cuuint64_t sb[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
@@ -893,7 +945,7 @@ namespace {
 
 bool same_conv(const ConvGeom &a, const ConvGeom &b) {
     return a.batch == b.batch && a.height == b.height && a.width == b.width && a.channels == b.channels &&
-           a.kh == b.kh && a.kw == b.kw && a.pad == b.pad;
+           a.kh == b.kh && a.kw == b.kw && a.pad == b.pad && a.nhwc_out == b.nhwc_out;
 }
 
 // Tile shape, shared-memory split, tensor maps and kernel variant for one product.
@@ -971,7 +1023,8 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
     // tiles.  Short walks are store-heavy and need no deep ring: they give stages up for staging tiles.
     const uint32_t avail = kSmemBudget + 1024;
     const uint32_t epi = short_walk && nt >= 3 ? 4u * (uint32_t)nt : 8u;
-    const uint32_t fixed = epi * kWideStageBytes + 256;
+    const bool nhwc = conv && conv->nhwc_out;                // transposed chunks need whole 4096-byte staging tiles
+    const uint32_t fixed = epi * (nhwc ? 2 * kWideStageBytes : kWideStageBytes) + 256;
     uint32_t stages = (avail - fixed) / p.stage_bytes;
     const uint32_t max_stages = p.stage_bytes <= 24 * 1024 ? (wlen <= 8 ? 6u : 7u) : (wlen <= 8 ? 4u : 8u);
     if (stages > max_stages) stages = max_stages;
@@ -983,7 +1036,8 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
     if (p.walk_cache) left -= cache_bytes;
     // staging per warp beyond the one 16-row tile already counted: two 32-row tiles, two 16-row tiles, or none
     const uint32_t unit = epi * kWideStageBytes;
-    if (left >= 3 * unit) { p.stg_bufs = 2; p.stg_tile_bytes = 2 * kWideStageBytes; }
+    if (nhwc) { p.stg_bufs = 1; p.stg_tile_bytes = 2 * kWideStageBytes; }
+    else if (left >= 3 * unit) { p.stg_bufs = 2; p.stg_tile_bytes = 2 * kWideStageBytes; }
     else if (left >= unit) { p.stg_bufs = 2; p.stg_tile_bytes = kWideStageBytes; }
     else { p.stg_bufs = 1; p.stg_tile_bytes = kWideStageBytes; }
     plan->smem = (size_t)stages * p.stage_bytes + (size_t)epi * p.stg_bufs * p.stg_tile_bytes + 256 +
@@ -996,7 +1050,8 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
     p.stg_swz_mask = 7;
     if (conv) {
         p.stg_swz_mask = (uint32_t)(p.cv_tw * (f32 ? 4 : 2)) / 16 - 1;      // 128 / 64 / 32 / 16-byte inner box of map_y
-        p.cv_plain = ((int64_t)conv->wo * (f32 ? 4 : 2)) % 16 != 0 || (ldy * (f32 ? 4 : 2)) % 16 != 0 ||
+        p.cv_nhwc = conv->nhwc_out;
+        p.cv_plain = (!p.cv_nhwc && ((int64_t)conv->wo * (f32 ? 4 : 2)) % 16 != 0) || (ldy * (f32 ? 4 : 2)) % 16 != 0 ||
                      reinterpret_cast<uintptr_t>(d_y) % 16 != 0;
         for (p.cv_tw_log2 = 0; (1 << p.cv_tw_log2) < p.cv_tw; ++p.cv_tw_log2) {}
         for (p.cv_img_log2 = 0; (1 << p.cv_img_log2) < p.cv_tw * p.cv_th; ++p.cv_img_log2) {}
@@ -1011,7 +1066,15 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
         const uint64_t yd[4] = {wo, ho, (uint64_t)conv->batch, (uint64_t)g.rows}, ys[3] = {wo * es, ho * wo * es, (uint64_t)ldy * es};
         const uint32_t yb[4] = {(uint32_t)p.cv_tw, (uint32_t)((f32 ? 32 : 64) / p.cv_tw), 1u, p.stg_tile_bytes / 128};
         if (p.cv_plain) my = CUtensorMap{};
-        else if (!make_map_4d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (int)es, d_y, yd, ys, yb))
+        else if (p.cv_nhwc) {
+            // Y [batch][ho][wo][ldy]: a chunk is {32 channels, tw, pixels / tw, 1}, laid out densely in the staging tile
+            const uint64_t nd[4] = {(uint64_t)g.rows, wo, ho, (uint64_t)conv->batch};
+            const uint64_t ns[3] = {(uint64_t)ldy * es, wo * (uint64_t)ldy * es, ho * wo * (uint64_t)ldy * es};
+            const uint32_t nb[4] = {32u, (uint32_t)p.cv_tw, (uint32_t)((f32 ? 32 : 64) / p.cv_tw), 1u};
+            if (!make_map_4d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (int)es, d_y, nd, ns, nb,
+                             /*swizzle=*/false))
+                return cudaErrorInvalidValue;
+        } else if (!make_map_4d(&my, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (int)es, d_y, yd, ys, yb))
             return cudaErrorInvalidValue;
     } else {
         p.x_map_3d = (ncols % kBoxN == 0) &&

@@ -159,7 +159,7 @@ bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const
 bool make_map_x3d(CUtensorMap *map, const void *base, uint64_t ncols, uint64_t k, uint64_t ldx, uint32_t bk, uint32_t nt);
 bool make_map_image(CUtensorMap *map, const void *image, uint64_t total_bytes, uint32_t entry_bytes);
 bool make_map_4d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *base, const uint64_t (&dims)[4],
-                 const uint64_t (&strides_bytes)[3], const uint32_t (&box)[4]);
+                 const uint64_t (&strides_bytes)[3], const uint32_t (&box)[4], bool swizzle = true);
 bool tensor_maps_available();
 
 }  // namespace tc

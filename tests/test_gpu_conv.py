@@ -136,3 +136,64 @@ def test_vgg_layer_matches_lowered_product_and_sampled_oracle(env):
         rows = np.arange(lo, hi)[inner]
         check_tolerance(yv[:, img, rows, :], ref[:, inner, :])
     L.close()
+
+
+NHWC_CASES = [
+    # s_out, kh, kw, pad, c, b, h, w, n, m, bm, keep
+    (96, 3, 3, 1, 64, 3, 12, 16, 2, 4, 32, 0.5),          # ragged rows of W (96 of 128), several pixel tiles
+    (200, 3, 3, 1, 64, 5, 9, 8, 1, 4, 128, 0.34),         # ragged in y, across images and in the channel blocks
+    (64, 5, 3, 1, 64, 2, 12, 16, 3, 4, 64, 0.6),          # dense-tile image
+    (128, 3, 3, 1, 128, 2, 28, 28, 1, 4, 64, 0.25),       # 28-pixel rows: fine in NHWC (the pixel pitch is what counts)
+    (100, 3, 3, 1, 64, 2, 10, 12, 2, 4, 32, 0.5),         # 100 channels: pixel pitch of 200 bytes, stored pixel by pixel
+]
+
+
+@pytest.mark.parametrize("s_out,kh,kw,pad,c,b,h,w,n,m,bm,keep", NHWC_CASES)
+@pytest.mark.parametrize("y_dtype", [0, 1])
+def test_conv_with_nhwc_output_matches_oracle(env, s_out, kh, kw, pad, c, b, h, w, n, m, bm, keep, y_dtype):
+    """Output channel fastest ([batch, ho, wo, rows]): the layout the next convolution reads."""
+    B, torch = env
+    wt, sal, act = conv_inputs(s_out, kh, kw, c, b, h, w, seed=s_out + 3 * h + w)
+    mk, vals, idx, wd, _wb = oracle_layer(wt, sal, n, m, bm, 64, keep)
+    ref = oracle.conv_fp64(wd, kh, kw, act, pad)                       # [s_out, b * ho * wo]
+    L = gpu_layer(B, torch, wt, sal, n, m, bm, 64, keep)
+    ho, wo = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    y = torch.full((b, ho, wo, s_out), 7.0, dtype=torch.float32 if y_dtype else torch.bfloat16, device="cuda")
+    guard = torch.full((64,), 7.0, dtype=y.dtype, device="cuda")        # allocated right after y
+    L.spmm_conv(bf16_dev(act, torch), kh, kw, pad, y=y, y_dtype=y_dtype, nhwc_out=True)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    got = y_to_f64(y.reshape(b * ho * wo, s_out), torch).T
+    check_tolerance(got, ref)
+    assert float(guard.float().min()) == 7.0 and float(guard.float().max()) == 7.0
+    L.close()
+
+
+def test_two_convolutions_chain_through_nhwc(env):
+    """VGG-16 stand-in conv2_1 -> conv2_2 (64 -> 128 -> 128 channels, 3 x 3, bias + ReLU fused, bf16 hand-over): the
+    first layer's NHWC output is the second layer's activation as it stands.  Each layer is checked against the
+    oracle's convolution of what it actually read."""
+    B, torch = env
+    b, h, w = 2, 56, 56
+    wt1, sal1, act = conv_inputs(128, 3, 3, 64, b, h, w, seed=21)
+    wt2, sal2, _ = conv_inputs(128, 3, 3, 128, 1, 4, 4, seed=22)
+    rng = np.random.default_rng(23)
+    bias1 = rng.standard_normal(128).astype(np.float32) * 0.1
+    bias2 = rng.standard_normal(128).astype(np.float32) * 0.1
+    _m1, _v1, _i1, wd1, _ = oracle_layer(wt1, sal1, 2, 4, 64, 64, 0.4)
+    _m2, _v2, _i2, wd2, _ = oracle_layer(wt2, sal2, 2, 4, 64, 64, 0.3)
+    L1 = gpu_layer(B, torch, wt1, sal1, 2, 4, 64, 64, 0.4)
+    L2 = gpu_layer(B, torch, wt2, sal2, 2, 4, 64, 64, 0.3)
+    from helpers import to_dev
+    L1.set_epilogue(to_dev(bias1, torch), relu=True)
+    L2.set_epilogue(to_dev(bias2, torch), relu=True)
+    y1 = L1.spmm_conv(bf16_dev(act, torch), 3, 3, 1, nhwc_out=True)            # [b, h, w, 128] bf16
+    y2 = L2.spmm_conv(y1, 3, 3, 1, nhwc_out=True)
+    torch.cuda.synchronize()
+    assert L1.device_status() == 0 and L2.device_status() == 0
+    ref1 = oracle.bias_relu(oracle.conv_fp64(wd1, 3, 3, act, 1), bias1, True)
+    check_tolerance(y_to_f64(y1.reshape(b * h * w, 128), torch).T, ref1)
+    y1_bits = y1.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)  # what the second layer read
+    ref2 = oracle.bias_relu(oracle.conv_fp64(wd2, 3, 3, y1_bits, 1), bias2, True)
+    check_tolerance(y_to_f64(y2.reshape(b * h * w, 128), torch).T, ref2)
+    L1.close(); L2.close()
