@@ -332,6 +332,44 @@ def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=50):
     return out
 
 
+def measure_two_addends(torch, B, dev, peaks, flush_l2, shared, iters=30):
+    """Patterns 2:4 cannot express in one pass (3:4, 4:8): the dense-tile image (default) against the same block
+    split into two 2:4-compliant addends that are multiplied into one accumulator by two sparse passes over the
+    same X tile.  Same tensor slots either way; the two-addend form moves 20 KB instead of 16 KB of weights per
+    block and, with 256-column tiles, has room for one accumulator only."""
+    d_s, d_w, d_x = shared
+    stream = torch.cuda.current_stream()
+    out = []
+    for (n, m, keep) in ((4, 8, 0.5), (4, 8, 0.25), (3, 4, 0.5), (3, 4, 0.25)):
+        layer = wl.sweep_cell(n, m, keep)
+        d_y = torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16, device=dev)
+        rec = {"workload": layer.name}
+        ys = {}
+        for kind in ("dense", "sparse2"):
+            os.environ["CRISP_EXEC_IMAGE"] = kind
+            L = B.HybridLayer(layer.rows, layer.k, n, m, layer.block_rows, layer.block_k, keep, device=dev)
+            L.build_mask(d_s).encode(d_w)
+            os.environ.pop("CRISP_EXEC_IMAGE")
+            ts = []
+            for i in range(3 + iters):
+                flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); L.spmm(d_x, y=d_y); b.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b) * 1e3)
+            ys[kind] = d_y.clone()
+            r = roofline_terms(L.bytes_model(layer.ncols), peaks, float(np.median(ts)) * 1e-3, layer.ncols)
+            rec[kind] = {"kernel": B.PATH_NAMES[L.last_launch()["path"]], "spmm_us": float(np.median(ts)),
+                         "spmm_us_min": float(np.min(ts)), "roofline_frac": r["frac"], "device_status": L.device_status()}
+            L.close()
+        d = (ys["dense"].float() - ys["sparse2"].float()).abs().max().item()
+        rec["max_abs_difference"] = d
+        rec["two_addends_over_dense"] = rec["sparse2"]["spmm_us"] / rec["dense"]["spmm_us"]
+        out.append(rec)
+    return out
+
+
 def summarise_cells(cells):
     """Per workload family: sum of our times, sum of the dense cuBLAS times, their ratio (layers with no kept
     block left out), and the spread of the roofline fraction."""
@@ -856,6 +894,7 @@ def run_ours(args, layer, rank, world):
         out["conv"] = measure_conv(torch, B, dev, peaks, flush_l2)
         out["saliency"] = measure_saliency(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
         out["pruning_iteration"] = measure_iteration(torch, B, dev, not args.no_cpu_baseline)
+        out["two_addend_form"] = measure_two_addends(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)

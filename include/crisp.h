@@ -95,6 +95,10 @@ typedef struct {
 #define CRISP_PATH_DIRECT 0   /* CUDA-core kernel on the canonical format (any shape)        */
 #define CRISP_PATH_DENSE  1   /* tcgen05 dense MMA over zero-expanded kept blocks            */
 #define CRISP_PATH_SPARSE 2   /* tcgen05 sparse (2:4) MMA over compressed kept blocks        */
+#define CRISP_PATH_SPARSE2 3  /* the same for patterns with up to four values per aligned 4-group
+                                 (3:4, 4:8, ...): the block is split into two 2:4-compliant addends,
+                                 both multiplied into one accumulator (opt-in, for measurements:
+                                 the dense-tile image is the default for those patterns)        */
 
 /* What the last crisp_spmm / crisp_spmm_conv on a handle really launched (crisp_last_launch).
  * `path` is the kernel family that ran, which differs from crisp_bytes_t.path when the operands

@@ -14,8 +14,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcrisp.so")
 
 OK, INVALID_ARG, UNSUPPORTED, BAD_SHAPE, BUFFER_TOO_SMALL, CUDA_ERROR, TIMEOUT = range(7)
-PATH_DIRECT, PATH_DENSE, PATH_SPARSE = 0, 1, 2
-PATH_NAMES = {0: "direct", 1: "dense_tcgen05", 2: "sparse_tcgen05"}
+PATH_DIRECT, PATH_DENSE, PATH_SPARSE, PATH_SPARSE2 = 0, 1, 2, 3
+PATH_NAMES = {0: "direct", 1: "dense_tcgen05", 2: "sparse_tcgen05", 3: "sparse_tcgen05_two_addends"}
 
 
 class LayerDesc(C.Structure):

@@ -53,12 +53,13 @@ int image_kind(const Geometry &g) {
     const char *e = std::getenv("CRISP_EXEC_IMAGE");
     if (e && !std::strcmp(e, "none")) return CRISP_PATH_DIRECT;
     if (e && !std::strcmp(e, "dense")) return CRISP_PATH_DENSE;
+    if (e && !std::strcmp(e, "sparse2") && !crisp::tc_pattern_is_sparse(g)) return CRISP_PATH_SPARSE2;
     return crisp::tc_pattern_is_sparse(g) ? CRISP_PATH_SPARSE : CRISP_PATH_DENSE;
 }
 
 size_t exec_payload_bytes(const Geometry &g, int kind) {
     if (kind == CRISP_PATH_DIRECT) return 0;
-    return crisp::tc_image_layout(g, kind == CRISP_PATH_SPARSE).total_bytes;
+    return crisp::tc_image_layout(g, kind).total_bytes;
 }
 
 size_t blk_col_bytes(const Geometry &g) { return align_up((size_t)g.nrt * g.kkeep * sizeof(int32_t) + 4); }
@@ -220,20 +221,20 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
     // 128-row blocks: one kept block is one tensor-core tile, so the encode kernel writes it directly
-    const bool fuse_tiles = h->exec_kind != CRISP_PATH_DIRECT && g.bm == 128;
+    const bool fuse_tiles = (h->exec_kind == CRISP_PATH_DENSE || h->exec_kind == CRISP_PATH_SPARSE) && g.bm == 128;
     crisp::TcImageLayout L = {};
-    if (h->exec_kind != CRISP_PATH_DIRECT) L = crisp::tc_image_layout(g, h->exec_kind == CRISP_PATH_SPARSE);
+    if (h->exec_kind != CRISP_PATH_DIRECT) L = crisp::tc_image_layout(g, h->exec_kind);
     // the walk lists of the tensor-core kernel depend on the mask only: CTAs of the encode kernel build them
     const bool tc = h->exec_kind != CRISP_PATH_DIRECT;
     crisp::WalkArgs walks = {};
-    if (tc) walks = crisp::tc_walk_args(g, h->exec_kind == CRISP_PATH_SPARSE, mask->d_blk_col, h->d_exec);
+    if (tc) walks = crisp::tc_walk_args(g, h->exec_kind, mask->d_blk_col, h->d_exec);
     if (e == cudaSuccess)
         e = crisp::launch_encode_canonical(d_w_bf16, ld_w, g, mask->d_blk_col, mask->d_nm_bits,
                                            h->d_blk_col, h->d_vals, h->d_idx, fuse_tiles ? h->exec_kind : 0,
                                            fuse_tiles ? h->d_exec + L.image_off : nullptr, L.a_bytes, L.entry_bytes,
                                            tc ? &walks : nullptr, st);
     if (e == cudaSuccess && tc)
-        e = crisp::launch_build_image(g, h->exec_kind == CRISP_PATH_SPARSE, h->d_blk_col, h->d_vals, h->d_idx,
+        e = crisp::launch_build_image(g, h->exec_kind, h->d_blk_col, h->d_vals, h->d_idx,
                                       h->d_exec, fuse_tiles, /*walks_done=*/true, st);
     if (e != cudaSuccess) { delete h; return CRISP_CUDA_ERROR; }
     *out = h;
@@ -280,7 +281,7 @@ crisp_status_t crisp_set_epilogue(crisp_handle_t h, const float *d_bias_f32, int
 crisp_status_t crisp_set_path(crisp_handle_t h, int32_t path) {
     if (!h) return CRISP_INVALID_ARG;
     if (path == -1 || path == CRISP_PATH_DIRECT) { h->forced_path = path; return CRISP_OK; }
-    if (path != CRISP_PATH_DENSE && path != CRISP_PATH_SPARSE) return CRISP_INVALID_ARG;
+    if (path != CRISP_PATH_DENSE && path != CRISP_PATH_SPARSE && path != CRISP_PATH_SPARSE2) return CRISP_INVALID_ARG;
     if (path != h->exec_kind) return CRISP_UNSUPPORTED;
     h->forced_path = path;
     return CRISP_OK;
@@ -301,7 +302,7 @@ crisp_status_t crisp_spmm(crisp_handle_t h, const uint16_t *d_x_bf16, int64_t ld
                                       d_y, ldy, y_dtype, h->epilogue, (cudaStream_t)stream);
         if (e == cudaSuccess) h->last = crisp_launch_info_t{CRISP_PATH_DIRECT, 0, 0, 1, 0, 0, 0, 0};
     } else {
-        e = crisp::launch_spmm_tc(h, path == CRISP_PATH_SPARSE, d_x_bf16, ldx, ncols, d_y, ldy, y_dtype, nullptr,
+        e = crisp::launch_spmm_tc(h, path, d_x_bf16, ldx, ncols, d_y, ldy, y_dtype, nullptr,
                                   (cudaStream_t)stream);
     }
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
@@ -329,7 +330,7 @@ crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, con
     if (!aligned(d_y, es)) return CRISP_INVALID_ARG;
     const int path = h->forced_path >= 0 ? h->forced_path : h->exec_kind;
     if (path == CRISP_PATH_DIRECT || h->g.kkeep == 0) return CRISP_UNSUPPORTED;
-    cudaError_t e = crisp::launch_spmm_tc(h, path == CRISP_PATH_SPARSE, d_act_nhwc, 0, ncols, d_y, ldy, y_dtype, &cg,
+    cudaError_t e = crisp::launch_spmm_tc(h, path, d_act_nhwc, 0, ncols, d_y, ldy, y_dtype, &cg,
                                           (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return CRISP_UNSUPPORTED;
     return e == cudaSuccess ? CRISP_OK : CRISP_CUDA_ERROR;
@@ -389,7 +390,8 @@ crisp_status_t crisp_bytes_model(crisp_handle_t h, int64_t ncols, int32_t y_dtyp
     out->x_bytes = touched_rows * ncols * 2;
     const int64_t elems = (int64_t)g.nrt * g.kkeep * g.bm * g.bk;
     out->path = h->forced_path >= 0 ? h->forced_path : h->exec_kind;
-    out->slot_macs = (out->path == CRISP_PATH_SPARSE ? elems / 2 : (out->path == CRISP_PATH_DENSE ? elems : g.nnz())) * ncols;
+    out->slot_macs = (out->path == CRISP_PATH_SPARSE ? elems / 2
+                      : (out->path == CRISP_PATH_DENSE || out->path == CRISP_PATH_SPARSE2 ? elems : g.nnz())) * ncols;
     return CRISP_OK;
 }
 

@@ -100,15 +100,16 @@ struct TcImageLayout {
     int wcap;               // capacity of one CTA tile's walk list (union of its row tiles' kept blocks)
     int stack;              // copies of the image, each shifted by 128 / stack rows (thin single-tile layers)
     uint32_t a_bytes;       // weight tile bytes per walk entry
-    uint32_t entry_bytes;   // weight tile + metadata
+    uint32_t entry_bytes;   // weight tile + metadata (two of each for the two-addend image)
+    int addends;            // sparse tiles per walk entry: 1, or 2 for the two-addend image
     size_t walk_col_off, walk_len_off, image_off, total_bytes;   // offsets inside the exec payload
 };
 bool tc_pattern_is_sparse(const Geometry &g);
-TcImageLayout tc_image_layout(const Geometry &g, bool sparse);
+TcImageLayout tc_image_layout(const Geometry &g, int kind);      // kind: CRISP_PATH_DENSE / SPARSE / SPARSE2
 // walk lists of the tensor-core kernel (walks.cuh): built by CTAs of the encode kernel (walks != nullptr in
 // launch_encode_canonical, then walks_done below) or by a kernel of their own
-struct WalkArgs tc_walk_args(const Geometry &g, bool sparse, const int32_t *d_mask_blk_col, uint8_t *d_exec);
-cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
+struct WalkArgs tc_walk_args(const Geometry &g, int kind, const int32_t *d_mask_blk_col, uint8_t *d_exec);
+cudaError_t launch_build_image(const Geometry &g, int kind, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, bool walks_done,
                                cudaStream_t st);
 bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int y_dtype, int64_t ncols);
@@ -116,7 +117,7 @@ bool tc_operands_ok(const void *x, int64_t ldx, const void *y, int64_t ldy, int 
 struct ConvGeom { int batch, height, width, channels, kh, kw, pad, ho, wo, nhwc_out; };
 // conv == nullptr: d_x is the [k, ncols] matrix.  Otherwise d_x is the activation and ncols = batch*ho*wo.
 // `h->plan` is reused when the operands, shape and epilogue are those of the previous call; `h->last` is filled in.
-cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols,
+cudaError_t launch_spmm_tc(crisp_handle_s *h, int kind, const uint16_t *d_x, int64_t ldx, int64_t ncols,
                            void *d_y, int64_t ldy, int y_dtype, const ConvGeom *conv, cudaStream_t st);
 // spmm_direct.cu
 cudaError_t launch_spmm_direct(const Geometry &g, const int32_t *d_blk_col, const uint16_t *d_vals,

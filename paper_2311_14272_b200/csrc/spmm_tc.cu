@@ -38,6 +38,8 @@ struct TcParams {
     int nst, wcap, bk, n_col_tiles, num_tiles, rows;
     int64_t ncols;
     uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
+    uint32_t addends;           // sparse tiles (each a_bytes + metadata) per walk entry: 2 when a block with up to four
+                                // values per aligned 4-group is multiplied as two 2:4-compliant addends
     uint32_t stg_bufs;          // staging tiles per epilogue warp (1, 2 or 4): stores in flight per warp
     uint32_t stg_tile_bytes;    // one staging tile: 16 or 32 rows of 128 bytes (= the row count of map_y's box)
     uint32_t stg_swz_mask;      // 16-byte chunk j of staging row r sits at j ^ (r & mask): 7 = 128-byte swizzle of
@@ -293,6 +295,15 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
                     mma_sparse(d_tmem, ad + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), accum | (uint32_t)j,
                                meta_tmem + (j & ~1));
                 meta_buf ^= 1u;
+                if (p.addends == 2) {               // second addend of the block: same X tile, same accumulator
+                    const uint32_t sub = (p.a_bytes + kMetaBytes) >> 4;
+                    const uint32_t meta2 = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                    tmem_copy_128x128b(meta2, m_desc0 + off + sub);
+#pragma unroll
+                    for (int j = 0; j < NM; ++j)
+                        mma_sparse(d_tmem, ad + sub + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), 1u, meta2 + (j & ~1));
+                    meta_buf ^= 1u;
+                }
             } else {
 #pragma unroll
                 for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * b_step, idesc, accum | (uint32_t)j);
@@ -617,7 +628,7 @@ __global__ void __launch_bounds__(256)
 build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16_t *__restrict__ vals,
                    const uint32_t *__restrict__ idx, int r, int nst, int wcap, int stack,
                    const int32_t *__restrict__ walk_col, const int32_t *__restrict__ walk_len, uint32_t a_bytes,
-                   uint32_t entry_bytes, uint8_t *__restrict__ image) {
+                   uint32_t entry_bytes, int addends, uint8_t *__restrict__ image) {
     extern __shared__ uint4 s_tile4[];
     uint8_t *tile = reinterpret_cast<uint8_t *>(s_tile4);
     __shared__ int s_blk[4];
@@ -678,15 +689,17 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
                 *reinterpret_cast<uint16_t *>(tile + (k >> 3) * 2048 + row * 16 + (k & 7) * 2) = vb[o];
             }
         } else {
-            // one thread per (local row, 4-group): at most two kept values by construction
+            // one thread per (local row, 4-group): at most two kept values per addend.  With one addend the pattern
+            // guarantees that; with two, the first two values (ascending position) go to the first addend and the
+            // rest to the second, each a 2:4-compliant tile with its own metadata, sub bytes apart.
             const int quads = g.bk / 4;
-            uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
+            const uint32_t sub = a_bytes + kMetaBytes;
             for (int item = threadIdx.x; item < g.bm * quads; item += blockDim.x) {
                 const int lr = item / quads, qd = item - lr * quads;
                 const int row = row0 + lr;
                 const int gi = (qd * 4) / g.m;
-                uint16_t v[2] = {0, 0};
-                int pos[2] = {0, 0}, cnt = 0;
+                uint16_t v4[4] = {0, 0, 0, 0};
+                int pos4[4] = {0, 0, 0, 0}, cnt4 = 0;
                 for (int vv = 0; vv < g.n; ++vv) {
                     const int o = (lr * groups + gi) * g.n + vv;
                     const int bit = o * g.idx_bits;
@@ -694,34 +707,44 @@ build_image_kernel(Geometry g, const int32_t *__restrict__ blk_col, const uint16
                     if ((bit & 31) + g.idx_bits > 32) t |= ib[(bit >> 5) + 1] << (32 - (bit & 31));
                     t &= field;
                     const int k = gi * g.m + (int)t;
-                    if ((k >> 2) == qd && cnt < 2) { v[cnt] = vb[o]; pos[cnt] = k & 3; ++cnt; }
+                    if ((k >> 2) == qd && cnt4 < 2 * addends) { v4[cnt4] = vb[o]; pos4[cnt4] = k & 3; ++cnt4; }
                 }
-                if (cnt == 0) { pos[0] = 0; pos[1] = 1; }
-                else if (cnt == 1) {
-                    if (pos[0] == 3) { v[1] = v[0]; v[0] = 0; pos[1] = 3; pos[0] = 0; }
-                    else pos[1] = 3;
+                for (int a = 0; a < addends; ++a) {
+                    uint16_t v[2] = {v4[2 * a], v4[2 * a + 1]};
+                    int pos[2] = {pos4[2 * a], pos4[2 * a + 1]};
+                    const int cnt = cnt4 - 2 * a < 0 ? 0 : (cnt4 - 2 * a > 2 ? 2 : cnt4 - 2 * a);
+                    if (cnt == 0) { v[0] = v[1] = 0; pos[0] = 0; pos[1] = 1; }
+                    else if (cnt == 1) {
+                        v[1] = 0;
+                        if (pos[0] == 3) { v[1] = v[0]; v[0] = 0; pos[1] = 3; pos[0] = 0; }
+                        else pos[1] = 3;
+                    }
+                    uint8_t *ta = tile + a * sub;
+                    uint32_t *meta = reinterpret_cast<uint32_t *>(ta + a_bytes);
+                    const int c0 = 2 * qd;                   // even: both slots share one 16-byte chunk
+                    *reinterpret_cast<uint32_t *>(ta + (c0 >> 3) * 2048 + row * 16 + (c0 & 7) * 2) =
+                        (uint32_t)v[0] | ((uint32_t)v[1] << 16);
+                    const uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
+                    const int k0 = qd * 4;
+                    const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
+                    atomicOr(&meta[lrow * 4 + (k0 >> 5)], nib << ((k0 & 15) + 16 * ((row >> 3) & 1)));
                 }
-                const int c0 = 2 * qd;                       // even: both slots share one 16-byte chunk
-                *reinterpret_cast<uint32_t *>(tile + (c0 >> 3) * 2048 + row * 16 + (c0 & 7) * 2) =
-                    (uint32_t)v[0] | ((uint32_t)v[1] << 16);
-                const uint32_t nib = (uint32_t)pos[0] | ((uint32_t)pos[1] << 2);
-                const int k0 = qd * 4;
-                const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
-                atomicOr(&meta[lrow * 4 + (k0 >> 5)], nib << ((k0 & 15) + 16 * ((row >> 3) & 1)));
             }
         }
     }
     if constexpr (kSparse) {
         // rows that carry no kept block here (row tiles that do not keep it, rows outside a stacked copy's
         // window) still need valid (distinct, ascending) index pairs
-        uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a_bytes);
-        for (int item = threadIdx.x; item < kTileM * (g.bk / 4); item += blockDim.x) {
-            const int row = item / (g.bk / 4), qd = item - row * (g.bk / 4);
-            const int sub = row >= shift ? (row - shift) / g.bm : r;
-            if (sub < r && s_blk[sub] >= 0) continue;
-            const int k0 = qd * 4;
-            const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
-            atomicOr(&meta[lrow * 4 + (k0 >> 5)], 0x4u << ((k0 & 15) + 16 * ((row >> 3) & 1)));
+        for (int a = 0; a < addends; ++a) {
+            uint32_t *meta = reinterpret_cast<uint32_t *>(tile + a * (a_bytes + kMetaBytes) + a_bytes);
+            for (int item = threadIdx.x; item < kTileM * (g.bk / 4); item += blockDim.x) {
+                const int row = item / (g.bk / 4), qd = item - row * (g.bk / 4);
+                const int sub_rt = row >= shift ? (row - shift) / g.bm : r;
+                if (sub_rt < r && s_blk[sub_rt] >= 0) continue;
+                const int k0 = qd * 4;
+                const int lrow = (row & 7) + 8 * ((k0 >> 4) & 1) + 16 * (row >> 4);
+                atomicOr(&meta[lrow * 4 + (k0 >> 5)], 0x4u << ((k0 & 15) + 16 * ((row >> 3) & 1)));
+            }
         }
     }
     __syncthreads();
@@ -857,8 +880,10 @@ bool tensor_maps_available() { return encode_tiled_fn() != nullptr; }
 
 bool tc_pattern_is_sparse(const Geometry &g) { return g.n <= 2; }   // <= 2 kept per aligned 4-group
 
-TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
+TcImageLayout tc_image_layout(const Geometry &g, int kind) {
+    const bool sparse = kind != CRISP_PATH_DENSE;
     TcImageLayout L;
+    L.addends = kind == CRISP_PATH_SPARSE2 ? 2 : 1;
     L.r = kTileM / g.bm;
     L.nst = (g.nrt + L.r - 1) / L.r;
     const int64_t cap = (int64_t)L.r * g.kkeep;
@@ -868,7 +893,7 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
     L.stack = 1;
     if (L.nst == 1 && g.bm < kTileM) L.stack = g.rows <= 32 ? 4 : (g.rows <= 64 ? 2 : 1);
     L.a_bytes = (uint32_t)(kTileM * g.bk * 2) / (sparse ? 2 : 1);
-    L.entry_bytes = L.a_bytes + (sparse ? kMetaBytes : 0);
+    L.entry_bytes = (uint32_t)L.addends * (L.a_bytes + (sparse ? kMetaBytes : 0));
     L.walk_col_off = 0;
     L.walk_len_off = align_up((size_t)L.nst * L.wcap * sizeof(int32_t) + 4);
     L.image_off = L.walk_len_off + align_up((size_t)L.nst * sizeof(int32_t) + 4);
@@ -876,8 +901,8 @@ TcImageLayout tc_image_layout(const Geometry &g, bool sparse) {
     return L;
 }
 
-WalkArgs tc_walk_args(const Geometry &g, bool sparse, const int32_t *d_blk_col, uint8_t *d_exec) {
-    const TcImageLayout L = tc_image_layout(g, sparse);
+WalkArgs tc_walk_args(const Geometry &g, int kind, const int32_t *d_blk_col, uint8_t *d_exec) {
+    const TcImageLayout L = tc_image_layout(g, kind);
     WalkArgs a;
     a.blk_col = d_blk_col;
     a.r = L.r; a.nst = L.nst; a.wcap = L.wcap;
@@ -887,15 +912,16 @@ WalkArgs tc_walk_args(const Geometry &g, bool sparse, const int32_t *d_blk_col, 
     return a;
 }
 
-cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_blk_col, const uint16_t *d_vals,
+cudaError_t launch_build_image(const Geometry &g, int kind, const int32_t *d_blk_col, const uint16_t *d_vals,
                                const uint32_t *d_idx, uint8_t *d_exec, bool tiles_done, bool walks_done,
                                cudaStream_t st) {
-    const TcImageLayout L = tc_image_layout(g, sparse);
+    const bool sparse = kind != CRISP_PATH_DENSE;
+    const TcImageLayout L = tc_image_layout(g, kind);
     if (g.nrt * g.kkeep == 0) return cudaSuccess;
     int32_t *walk_col = reinterpret_cast<int32_t *>(d_exec + L.walk_col_off);
     int32_t *walk_len = reinterpret_cast<int32_t *>(d_exec + L.walk_len_off);
     uint8_t *image = d_exec + L.image_off;
-    if (!walks_done) build_walks_kernel<<<L.nst, 256, 0, st>>>(g, tc_walk_args(g, sparse, d_blk_col, d_exec));
+    if (!walks_done) build_walks_kernel<<<L.nst, 256, 0, st>>>(g, tc_walk_args(g, kind, d_blk_col, d_exec));
     if (tiles_done) return cudaGetLastError();       // the encode kernel already wrote the weight tiles
     const int grid = L.stack * L.nst * L.wcap;
     const size_t smem_img = (size_t)L.entry_bytes + (size_t)g.vals_per_block() * 2 + (size_t)(g.vals_per_block() * g.idx_bits / 32) * 4 + 16;
@@ -906,10 +932,10 @@ cudaError_t launch_build_image(const Geometry &g, bool sparse, const int32_t *d_
     }
     if (sparse)
         build_image_kernel<true><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.nst, L.wcap, L.stack, walk_col,
-                                                                    walk_len, L.a_bytes, L.entry_bytes, image);
+                                                                    walk_len, L.a_bytes, L.entry_bytes, L.addends, image);
     else
         build_image_kernel<false><<<grid, 256, smem_img, st>>>(g, d_blk_col, d_vals, d_idx, L.r, L.nst, L.wcap, L.stack, walk_col,
-                                                                     walk_len, L.a_bytes, L.entry_bytes, image);
+                                                                     walk_len, L.a_bytes, L.entry_bytes, L.addends, image);
     return cudaGetLastError();
 }
 
@@ -949,12 +975,13 @@ bool same_conv(const ConvGeom &a, const ConvGeom &b) {
 }
 
 // Tile shape, shared-memory split, tensor maps and kernel variant for one product.
-cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y,
+cudaError_t make_plan(const crisp_handle_s *h, int kind, const uint16_t *d_x, int64_t ldx, int64_t ncols, void *d_y,
                       int64_t ldy, int y_dtype, const ConvGeom *conv, int device, TcPlan *plan) {
     const Geometry &g = h->g;
     const uint8_t *d_exec = h->d_exec;
     const int nt_override = h->nt_override;
-    const TcImageLayout L = tc_image_layout(g, sparse);
+    const bool sparse = kind != CRISP_PATH_DENSE;
+    const TcImageLayout L = tc_image_layout(g, kind);
     const int sm_count = sm_count_of(device);
     // column tile: 4 boxes (256 columns).  For the sparse image that leaves room for one accumulator
     // only (256 + 8 metadata columns), which still beats 3 boxes with two accumulators: the kernel is
@@ -1015,7 +1042,7 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
     const int64_t tiles = (int64_t)p.n_col_tiles * L.nst;
     if (tiles > 0x7FFFFFFF) return cudaErrorInvalidValue;
     p.num_tiles = (int)tiles;
-    p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes;
+    p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes; p.addends = (uint32_t)L.addends;
     p.box_bytes = (uint32_t)(kBoxN * g.bk * 2);
     p.stage_bytes = p.entry_bytes + nt * p.box_bytes;
     // Shared memory (the whole 227 KB; the base is 1024-aligned): the ring gets as many stages as fit next
@@ -1121,7 +1148,7 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
 #undef CRISP_TC_VARIANT_E
 #undef CRISP_TC_VARIANT_C
     crisp_launch_info_t &info = plan->info;
-    info.path = sparse ? CRISP_PATH_SPARSE : CRISP_PATH_DENSE;
+    info.path = kind;
     info.tile_cols = nt * kBoxN;
     info.accumulators = acc;
     info.stack = stack;
@@ -1134,7 +1161,7 @@ cudaError_t make_plan(const crisp_handle_s *h, bool sparse, const uint16_t *d_x,
 
 }  // namespace
 
-cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, int64_t ldx, int64_t ncols,
+cudaError_t launch_spmm_tc(crisp_handle_s *h, int kind, const uint16_t *d_x, int64_t ldx, int64_t ncols,
                            void *d_y, int64_t ldy, int y_dtype, const ConvGeom *conv, cudaStream_t st) {
     int device = 0;
     cudaError_t e = cudaGetDevice(&device);
@@ -1146,7 +1173,7 @@ cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, 
                      plan->device == device && plan->skip_stage == h->debug_skip_stage &&
                      plan->wait_limit == h->wait_limit_cycles && plan->has_conv == (conv != nullptr) &&
                      (!conv || same_conv(plan->conv, *conv)) && plan->p.status == h->d_status &&
-                     plan->info.path == (sparse ? CRISP_PATH_SPARSE : CRISP_PATH_DENSE);
+                     plan->info.path == kind;
     if (!hit) {
         if (!plan) {
             plan = new (std::nothrow) TcPlan;
@@ -1154,7 +1181,7 @@ cudaError_t launch_spmm_tc(crisp_handle_s *h, bool sparse, const uint16_t *d_x, 
             h->plan = plan;
         }
         plan->x = nullptr;                                  // not valid until the plan below is complete
-        e = make_plan(h, sparse, d_x, ldx, ncols, d_y, ldy, y_dtype, conv, device, plan);
+        e = make_plan(h, kind, d_x, ldx, ncols, d_y, ldy, y_dtype, conv, device, plan);
         if (e != cudaSuccess) return e;
         plan->x = d_x; plan->y = d_y; plan->bias = h->epilogue.bias;
         plan->ldx = ldx; plan->ldy = ldy; plan->ncols = ncols;

@@ -60,7 +60,8 @@ CASES = [
 
 # which execution image crisp_encode lays out: the default choice (2:4 sparse MMA when n <= 2, dense
 # tiles otherwise), dense tiles forced, or none (CUDA-core kernel on the canonical format)
-IMAGES = ["auto", "dense", "none"]
+# "sparse2": patterns with more than two values per 4-group as two 2:4-compliant addends (others: the default image)
+IMAGES = ["auto", "dense", "none", "sparse2"]
 
 
 @pytest.fixture(params=IMAGES)
@@ -78,6 +79,8 @@ def expected_path(B, image, n, kkeep=1):
         return B.PATH_DIRECT
     if image == "dense":
         return B.PATH_DENSE
+    if image == "sparse2" and n > 2:
+        return B.PATH_SPARSE2
     return B.PATH_SPARSE if n <= 2 else B.PATH_DENSE
 
 
