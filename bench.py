@@ -909,6 +909,72 @@ def run_ours(args, layer, rank, world):
         dist.destroy_process_group()
 
 
+def render_markdown(d):
+    """Markdown tables of one JSON line of this program (the tables of the benchmark spec are this output)."""
+    o = []
+    r, ph, c = d["roofline"], d["phases"], d["config"]
+    o.append(f"Headline step ({c['workload']}, {c['rows']}x{c['k']}x{c['ncols']}, block {c['block'][0]}x{c['block'][1]}, "
+             f"kkeep {c['kkeep']}): `value` {d['value']:.1f} useful TFLOP/s, `ms_per_step` {d['ms_per_step'] * 1e3:.1f} us "
+             f"(`phases`: mask {ph['mask_us']:.1f}, encode {ph['encode_us']:.1f}, SpMM {ph['spmm_us']:.1f} us; "
+             f"{d['steps']} steps, L2 flushed before each).")
+    o.append(f"`roofline`: bound {r['bound']}, kernel {r['kernel']}, `t_kernel_us` {r['t_kernel_us']:.1f} (median "
+             f"{r['t_kernel_median_us']:.1f}, min {r['t_kernel_min_us']:.1f}; back to back {r['t_kernel_back_to_back_us']:.1f}), "
+             f"`t_tensor_us` {r['t_tensor_us']:.1f}, `t_hbm_us` {r['t_hbm_us']:.1f}, `frac` {r['frac']:.3f} "
+             f"(back to back {r['frac_back_to_back']:.3f}) {r['peak_kind']}, `speedup_vs_dense_cublas` "
+             f"{r['speedup_vs_dense_cublas']:.2f} (dense {r['dense_cublas_us']:.1f} us), `traffic` {r['traffic']}.")
+    e, ei = d["e2e"], d["e2e_inference"]
+    o.append(f"`e2e` (S, W, X in and Y out every step): {e['ms_per_step']:.2f} ms, {e['value']:.1f} TFLOP/s "
+             f"(one stream: {e['serial_ms_per_step']:.2f} ms); `e2e_inference` (handle resident, X in, Y out): "
+             f"{ei['ms_per_step']:.2f} ms, {ei['value']:.1f} TFLOP/s.")
+    if "cpu_baseline" in d:
+        cb = d["cpu_baseline"]
+        o.append(f"`cpu_baseline` (oracle, {cb['cores']} host cores, {cb['sample']}): {cb['value']:.4f} TFLOP/s.")
+    cells = d.get("cells", [])
+
+    def row(x):
+        fr = "-" if x["roofline_frac"] is None else f"{x['roofline_frac']:.2f} / {x['roofline_frac_literal']:.2f}"
+        return (f"| {x['workload']} | {x['rows']}x{x['k']}x{x['ncols']} | {x['nm']} | {x['kkeep']} | {x['kernel'].replace('_tcgen05', '')} "
+                f"{x['tile_cols']}c/{x['accumulators']}a{'/s' + str(x['stack']) if x['stack'] > 1 else ''} | {x['spmm_us']:.1f} ({x['spmm_us_min']:.1f}) | "
+                f"{x['spmm_warm_us']:.1f} | {x['dense_cublas_us']:.1f} | {x['speedup_vs_dense_cublas']:.2f} | "
+                f"{x['useful_tflops']:.1f} | {fr} |")
+
+    head = ("| workload | rows x k x ncols | N:M | kkeep | kernel (tile columns / accumulators) | SpMM us cold: median (min) | warm | "
+            "dense cuBLAS us | x dense | useful TFLOP/s | roofline slot-aware / literal |\n|---|---|---|---|---|---|---|---|---|---|---|")
+    for cfg, title in ((5, "Sweep (config 5) and 3:4"), (1, "Config 1"), (2, "Config 2"), (3, "Config 3: VGG-16 stand-in"),
+                       (4, "Config 4: MobileNetV2 stand-in")):
+        rows = [x for x in cells if x["config"] == cfg]
+        if rows:
+            o.append(f"\n**{title}** (`cells`)\n\n" + head + "\n" + "\n".join(row(x) for x in rows))
+    if "summary" in d:
+        o.append("\n**Per family** (`summary`; layers without a kept block left out)\n\n| family | layers | ours us | dense cuBLAS us | x dense | "
+                 "useful TFLOP/s | roofline min / median / max | faster than dense |\n|---|---|---|---|---|---|---|---|")
+        for k, v in d["summary"].items():
+            if "spmm_us_sum" in v:
+                o.append(f"| {k} | {v['layers']} | {v['spmm_us_sum']:.1f} | {v['dense_cublas_us_sum']:.1f} | {v['speedup_vs_dense_cublas']:.2f} | "
+                         f"{v['useful_tflops']:.1f} | {v['roofline_frac_min']:.2f} / {v['roofline_frac_median']:.2f} / {v['roofline_frac_max']:.2f} | "
+                         f"{v['faster_than_dense']} of {v['layers']} |")
+        lo = d["summary"]["sweep_keep_le_0.5"]
+        o.append(f"\nSweep cells with keep <= 0.5: {lo['at_or_above_60pct_of_roofline']} of {lo['cells']} at or above 0.60 of the "
+                 f"slot-aware roofline, {lo['faster_than_dense']} of {lo['cells']} faster than dense cuBLAS.")
+    for t in d.get("two_addend_form", []):
+        o.append(f"`two_addend_form` {t['workload']}: dense tiles {t['dense']['spmm_us']:.1f} us, two 2:4 addends "
+                 f"{t['sparse2']['spmm_us']:.1f} us ({t['two_addends_over_dense']:.2f}x), max |difference| {t['max_abs_difference']:.4f}.")
+    for t in d.get("pruning_iteration", []):
+        o.append(f"`pruning_iteration` {t['network']}: {t['layers']} layers, {t['weights']} weights, {t['samples']} gradient samples, "
+                 f"{t['iteration_us']:.0f} us per iteration ({t['launches']} launches), oracle {t.get('oracle_us', 0) / 1e3:.0f} ms, "
+                 f"kept counts equal: {t.get('matches_oracle')}.")
+    for t in d.get("global_rank", []):
+        o.append(f"`global_rank` {t['network']}: {t['global_rank_us']:.1f} us ({t['rank_positions']} rank positions), oracle "
+                 f"{t.get('oracle_us', 0):.0f} us, equal: {t.get('matches_oracle')}.")
+    for t in d.get("conv", []):
+        o.append(f"`conv` {t['workload']} {t['activation']}: gather {t['conv_us']:.1f} us, lowered product {t['lowered_spmm_us']:.1f}, "
+                 f"dense cuBLAS on the lowered matrix {t['dense_cublas_lowered_us']:.1f}; identical to lowered: {t['identical_to_lowered']}.")
+    if "saliency" in d:
+        t = d["saliency"]
+        o.append(f"`saliency` {t['workload']}: {t['us']:.1f} us, {t['achieved_gbs']:.0f} GB/s = {t['roofline_frac']:.2f} of the HBM peak.")
+    return "\n".join(o)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -921,7 +987,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cells", action="store_true", help="skip the per-layer / per-cell SpMM timings")
     ap.add_argument("--cell-iters", type=int, default=50, help="timed launches per cell and protocol")
+    ap.add_argument("--render", metavar="JSON_FILE", help="print the markdown tables of a stored JSON line and exit")
     args = ap.parse_args()
+    if args.render:
+        print(render_markdown(json.loads([l for l in open(args.render) if l.startswith("{")][-1])))
+        return
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     layer = pick_layer(args.workload)
