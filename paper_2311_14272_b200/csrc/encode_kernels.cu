@@ -151,6 +151,123 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
     }
 }
 
+// Fast path of encode_block_kernel for groups of 4 with one or two kept values (1:4, 2:4) and blocks 64 or 128
+// elements deep, which is what the large layers use.  Everything a 4-group needs follows from its four mask
+// bits, so it is looked up: a 16-entry table (built per CTA) gives, per nibble, the byte-permute selector that
+// picks the two kept bf16 values out of the group's two registers, which of the two slots carry a value, the 2:4
+// metadata nibble and the offset field.  Values, offsets, tile slots and metadata are then assembled in
+// registers, combined across the lanes that share a 32-bit word with shuffles, and stored once: no shared-memory
+// atomics, no zero-filling, a fraction of the instructions of the general kernel (which was bound by instruction
+// issue).  Rows are visited so that rows r and r + 8 (whose metadata shares words) sit in the same warp.
+// Output identical to encode_block_kernel's.  TILE: 0 or CRISP_PATH_SPARSE (128-row blocks).
+template <int N, int TILE>
+__global__ void __launch_bounds__(256, 8)
+encode_block_m4_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, const int32_t *__restrict__ mask_blk_col,
+                       const uint32_t *__restrict__ nm_bits, int32_t *__restrict__ blk_col, uint16_t *__restrict__ vals,
+                       uint32_t *__restrict__ idx, uint8_t *__restrict__ image, uint32_t a_bytes, uint32_t entry_bytes,
+                       WalkArgs walks) {
+    extern __shared__ uint32_t s_buf[];
+    __shared__ uint32_t s_lut[16], s_lut_mask[16];
+    if ((int)blockIdx.x < walks.nctas) {
+        __shared__ WalkShared s_walks;
+        build_walks_body(g, walks, blockIdx.x, s_walks);
+        return;
+    }
+    if (threadIdx.x < 16) {
+        // nibble -> slots (a, b), their validity, metadata nibble, first kept position
+        const uint32_t nib = threadIdx.x;
+        int a = 0, b = 1, va = 0, vb = 0, first = 0;
+        if (nib) {
+            first = __ffs(nib) - 1;
+            const uint32_t rest = nib & (nib - 1);
+            if (rest) { a = first; va = 1; b = __ffs(rest) - 1; vb = 1; }
+            else if (first == 3) { a = 0; b = 3; vb = 1; }
+            else { a = first; va = 1; b = 3; }
+        }
+        const uint32_t sel = (uint32_t)(2 * a) | ((uint32_t)(2 * a + 1) << 4) | ((uint32_t)(2 * b) << 8) | ((uint32_t)(2 * b + 1) << 12);
+        s_lut[nib] = sel | ((uint32_t)(a | (b << 2)) << 16) | ((uint32_t)first << 20);
+        s_lut_mask[nib] = (va ? 0x0000FFFFu : 0u) | (vb ? 0xFFFF0000u : 0u);
+    }
+    const int blk = (int)blockIdx.x - walks.nctas;    // rt * kkeep + slot
+    const int rt = blk / g.kkeep;
+    const int jb = mask_blk_col[blk];
+    const int groups = g.bk / 4;
+    const int vpb = g.bm * groups * N;
+    const int idx_words = vpb * 2 / 32;
+    const int val_words = vpb / 2;
+    uint32_t *s_idx = s_buf;                                                        // [idx_words]
+    uint32_t *s_val32 = s_buf + idx_words;                                          // [vpb / 2]
+    uint8_t *tile = reinterpret_cast<uint8_t *>(s_buf + idx_words + (vpb + 7) / 8 * 4);   // [entry_bytes], 16-byte aligned
+    if (threadIdx.x == 0) blk_col[blk] = jb;
+    if constexpr (TILE == CRISP_PATH_SPARSE)           // metadata words beyond block_k / 32 per row are never written
+        for (uint32_t i = threadIdx.x; i < (entry_bytes - a_bytes) / 16; i += blockDim.x)
+            reinterpret_cast<uint4 *>(tile + a_bytes)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    const int L = g.bk / 8;                            // 16-byte loads per row: 8 or 16
+    const int lshift = L == 8 ? 3 : 4;
+    for (int li = threadIdx.x; li < g.bm * L; li += blockDim.x) {
+        const int q = li >> lshift, c8 = li & (L - 1);
+        const int r = ((q & 1) << 3) | ((q >> 1) & 7) | (q & ~15);      // rows q, q ^ 1 of the walk are r, r ^ 8
+        const int64_t row = (int64_t)rt * g.bm + r;
+        const int64_t col8 = (int64_t)jb * g.bk + (int64_t)c8 * 8;
+        uint32_t wv[4] = {0u, 0u, 0u, 0u};
+        if (row < g.rows && col8 + 8 <= g.k) {
+            const uint4 t = __ldg(reinterpret_cast<const uint4 *>(w + row * ld + col8));
+            wv[0] = t.x; wv[1] = t.y; wv[2] = t.z; wv[3] = t.w;
+        } else if (row < g.rows && col8 < g.k) {
+            uint16_t v8[8];
+            load_group<8>(w, ld, g.rows, g.k, row, col8, false, v8);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) wv[i] = (uint32_t)v8[2 * i] | ((uint32_t)v8[2 * i + 1] << 16);
+        }
+        const uint32_t bits8 = (nm_bits[row * g.wpr + (col8 >> 5)] >> (col8 & 31)) & 0xFFu;
+        const uint32_t e0 = s_lut[bits8 & 15u], e1 = s_lut[bits8 >> 4];
+        const uint32_t p0 = __byte_perm(wv[0], wv[1], e0 & 0xFFFFu) & s_lut_mask[bits8 & 15u];
+        const uint32_t p1 = __byte_perm(wv[2], wv[3], e1 & 0xFFFFu) & s_lut_mask[bits8 >> 4];
+        const int item0 = r * groups + 2 * c8;                          // the thread's two groups: item0, item0 + 1
+        if constexpr (TILE == CRISP_PATH_SPARSE) {
+            // slot pairs of the two 4-groups: compressed columns 4 * c8 .. 4 * c8 + 3, one 8-byte store
+            *reinterpret_cast<uint2 *>(tile + (c8 >> 1) * 2048 + r * 16 + (c8 & 1) * 8) = make_uint2(p0, p1);
+            // metadata: this thread's two nibbles, the neighbour's (other half of the 16-element chunk) and those
+            // of row r ^ 8 make one 32-bit word
+            uint32_t mv = (((e0 >> 16) & 15u) | (((e1 >> 16) & 15u) << 4)) << (8 * (c8 & 1) + 16 * (q & 1));
+            mv |= __shfl_xor_sync(0xFFFFFFFFu, mv, 1);
+            mv |= __shfl_xor_sync(0xFFFFFFFFu, mv, L);
+            if (((c8 | q) & 1) == 0) {
+                const int lrow = (r & 7) + 8 * ((c8 >> 1) & 1) + 16 * (r >> 4);
+                reinterpret_cast<uint32_t *>(tile + a_bytes)[lrow * 4 + (c8 >> 2)] = mv;
+            }
+        }
+        if constexpr (N == 2) {
+            // both values of a group are kept values in ascending position: the slot pair is the canonical pair
+            *reinterpret_cast<uint2 *>(s_val32 + item0) = make_uint2(p0, p1);
+            uint32_t f = (((e0 >> 16) & 15u) | (((e1 >> 16) & 15u) << 4)) << (8 * (c8 & 3));
+            f |= __shfl_xor_sync(0xFFFFFFFFu, f, 1);
+            f |= __shfl_xor_sync(0xFFFFFFFFu, f, 2);
+            if ((c8 & 3) == 0) s_idx[(item0 >> 3)] = f;                  // 4 bits per group: 8 groups per word
+        } else {
+            // one kept value per group: it sits in slot 0, or in slot 1 when it is the group's last element
+            const uint32_t v0 = (p0 & 0xFFFFu) | (p0 >> 16), v1 = (p1 & 0xFFFFu) | (p1 >> 16);
+            s_val32[item0 >> 1] = v0 | (v1 << 16);
+            uint32_t f = (((e0 >> 20) & 3u) | (((e1 >> 20) & 3u) << 2)) << (4 * (c8 & 7));
+            f |= __shfl_xor_sync(0xFFFFFFFFu, f, 1);
+            f |= __shfl_xor_sync(0xFFFFFFFFu, f, 2);
+            f |= __shfl_xor_sync(0xFFFFFFFFu, f, 4);
+            if ((c8 & 7) == 0) s_idx[(item0 >> 4)] = f;                  // 2 bits per group: 16 groups per word
+        }
+    }
+    __syncthreads();
+    uint32_t *vout = reinterpret_cast<uint32_t *>(vals + (int64_t)blk * vpb);
+    for (int i = threadIdx.x; i < val_words; i += blockDim.x) vout[i] = s_val32[i];
+    uint32_t *iout = idx + (int64_t)blk * idx_words;
+    for (int i = threadIdx.x; i < idx_words; i += blockDim.x) iout[i] = s_idx[i];
+    if constexpr (TILE != 0) {
+        uint4 *out = reinterpret_cast<uint4 *>(image + (int64_t)blk * entry_bytes);
+        for (uint32_t i = threadIdx.x; i < entry_bytes / 16; i += blockDim.x) out[i] = reinterpret_cast<uint4 *>(tile)[i];
+    }
+}
+
 __global__ void __launch_bounds__(256)
 decode_block_kernel(Geometry g, const int32_t *__restrict__ blk_col,
                     const uint16_t *__restrict__ vals, const uint32_t *__restrict__ idx,
@@ -203,7 +320,22 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
         kern<<<nblocks + wa.nctas, 256, smem, st>>>(d_w, ld, g, vec_ok, d_mask_blk_col, d_nm_bits, d_blk_col, \
                                                      d_vals, d_idx, d_image, a_bytes, entry_bytes, wa);      \
     } while (0)
-    if (g.m == 4) {
+    // groups of 4 with one or two kept values, 64- or 128-deep blocks, 16-byte aligned rows: the table-driven kernel
+    const bool fast = g.m == 4 && g.n <= 2 && (g.bk == 64 || g.bk == 128) && vec_ok && tile_kind != CRISP_PATH_DENSE;
+#define CRISP_ENCODE_FAST(NV, TV)                                                                            \
+    do {                                                                                                     \
+        auto kern = encode_block_m4_kernel<NV, TV>;                                                          \
+        if (smem > 48 * 1024) {                                                                              \
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            if (e != cudaSuccess) return e;                                                                  \
+        }                                                                                                    \
+        kern<<<nblocks + wa.nctas, 256, smem, st>>>(d_w, ld, g, d_mask_blk_col, d_nm_bits, d_blk_col, d_vals,  \
+                                                    d_idx, d_image, a_bytes, entry_bytes, wa);               \
+    } while (0)
+    if (fast) {
+        if (g.n == 2) { if (tile_kind == CRISP_PATH_SPARSE) CRISP_ENCODE_FAST(2, CRISP_PATH_SPARSE); else CRISP_ENCODE_FAST(2, 0); }
+        else { if (tile_kind == CRISP_PATH_SPARSE) CRISP_ENCODE_FAST(1, CRISP_PATH_SPARSE); else CRISP_ENCODE_FAST(1, 0); }
+    } else if (g.m == 4) {
         if (tile_kind == CRISP_PATH_SPARSE) CRISP_ENCODE_LAUNCH(4, CRISP_PATH_SPARSE);
         else if (tile_kind == CRISP_PATH_DENSE) CRISP_ENCODE_LAUNCH(4, CRISP_PATH_DENSE);
         else CRISP_ENCODE_LAUNCH(4, 0);
@@ -213,6 +345,7 @@ cudaError_t launch_encode_canonical(const uint16_t *d_w, int64_t ld, const Geome
         else CRISP_ENCODE_LAUNCH(8, 0);
     }
 #undef CRISP_ENCODE_LAUNCH
+#undef CRISP_ENCODE_FAST
     return cudaGetLastError();
 }
 
