@@ -1,8 +1,8 @@
 // Tensor-core SpMM over kept blocks (sm_100a): TMA-staged, warp-specialised, tcgen05 MMA with
 // TMEM accumulators.  Sec. III-E of the paper, mapped onto B200:
-//   step 1 (load the activations of kept blocks): the producer warp walks the kept-block list of
-//           a 128-row tile and issues, per kept block, one bulk copy of the weight tile (from the
-//           execution image) and TMA tensor loads of the X rows [blk_col*Bk, +Bk) only;
+//   step 1 (load the activations of kept blocks): two producer threads walk the kept-block list of
+//           a 128-row tile; per kept block one issues a tiled copy of the weight tile (from the
+//           execution image), the other TMA tensor loads of the X rows [blk_col*Bk, +Bk) only;
 //   step 2 (select activations by offset): either the 2:4 metadata drives tcgen05.mma.sp's operand
 //           selection (sparse image), or the weight tile is stored zero-expanded so that the
 //           selection is the identity (dense image);
@@ -65,7 +65,7 @@ struct TcParams {
     const float *bias;          // layer epilogue: Y = act(W*X + bias); nullptr = no bias
     int relu;
     unsigned long long wait_limit;   // cycles after which a wait gives up and the kernel reports CRISP_TIMEOUT
-    int skip_fill;              // test hook (-1 = off): the producer leaves out the loads of its skip_fill-th pipeline
+    int skip_fill;              // test hook (-1 = off): the producers leave out the loads of the skip_fill-th pipeline
                                 // fill, so that the wait for it runs into wait_limit
     int a_map;                  // map_a views the image as rows of 256 bytes: weight tiles come in as tiled loads
     int x_map_3d;               // map_x views X as [ncols/64][k][64]: one load fetches all NT boxes
@@ -73,7 +73,7 @@ struct TcParams {
 
 constexpr uint32_t kWideStageBytes = 2048;                      // epilogue staging tile: 16 rows x 128 bytes
 // Epilogue warps: two per TMEM lane quarter, or four where short walks make the epilogue the longest role.
-// Threads: warp 0 producer, warp 1 MMA issuer, then the epilogue warps.
+// Threads: warp 0 weight-tile producer, warp 1 MMA issuer, the epilogue warps, then one warp as the X producer.
 
 // Where a tile's columns start: the first column (matrix mode) or the first output pixel (x, y, image) of
 // the tile's box (convolution mode).
@@ -329,7 +329,7 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
 // X box layout: TMA SWIZZLE_128B, 64 columns (128 bytes) x bk rows; MN-major operand with 1024 bytes
 // between 8-row K groups and box_bytes between 64-column groups.
 template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi, bool kConv>
-__global__ void __launch_bounds__(64 + 32 * kEpi, 1)
+__global__ void __launch_bounds__(96 + 32 * kEpi, 1)
 spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                const __grid_constant__ CUtensorMap map_a, TcParams p) {
     constexpr int kTileN = NT * kBoxN;
@@ -357,26 +357,32 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // walk would otherwise spend two dependent global loads per tile in the producer's serial loop.
     int32_t *s_walk = reinterpret_cast<int32_t *>(ctrl_gen + 256);
 
+    // Set-up, ordered so that its round trips run side by side: warp 1 asks for tensor memory at once, every
+    // thread asks for its first word of the walk lists before thread 0 builds the barriers, and the words are
+    // stored to shared memory afterwards.
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < p.num_stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kEpi); }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        prefetch_tensormap(&map_x);
-        prefetch_tensormap(&map_a);
-        if (!(kConv && p.cv_plain)) prefetch_tensormap(&map_y);
-    }
-    if (p.walk_cache) {
-        for (int i = threadIdx.x; i < p.nst; i += blockDim.x) s_walk[i] = p.walk_len[i];
-        for (int i = threadIdx.x; i < p.nst * p.wcap; i += blockDim.x) s_walk[p.nst + i] = p.walk_col[i];
-    }
-    const int32_t *walk_len = p.walk_cache ? s_walk : p.walk_len;
-    const int32_t *walk_col = p.walk_cache ? s_walk + p.nst : p.walk_col;
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_base_slot)), kTmemCols);
         tmem_relinquish();
     }
+    const int walk_words = p.walk_cache ? p.nst * (p.wcap + 1) : 0;     // [nst] lengths, then [nst][wcap] columns
+    int32_t walk_w0 = 0;
+    if ((int)threadIdx.x < walk_words)
+        walk_w0 = (int)threadIdx.x < p.nst ? p.walk_len[threadIdx.x] : p.walk_col[(int)threadIdx.x - p.nst];
+    if (threadIdx.x == 0) {
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_x);
+        if (!(kConv && p.cv_plain)) prefetch_tensormap(&map_y);
+        for (uint32_t s = 0; s < p.num_stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int a = 0; a < kAccStages; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, kEpi); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if ((int)threadIdx.x < walk_words) s_walk[threadIdx.x] = walk_w0;
+    for (int i = threadIdx.x + blockDim.x; i < walk_words; i += blockDim.x)
+        s_walk[i] = i < p.nst ? p.walk_len[i] : p.walk_col[i - p.nst];
+    const int32_t *walk_len = p.walk_cache ? s_walk : p.walk_len;
+    const int32_t *walk_col = p.walk_cache ? s_walk + p.nst : p.walk_col;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -386,79 +392,94 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // Both single-thread roles below are bound by their own dependent-instruction latency (one warp per
     // scheduler, ~5 cycles per dependent instruction), so their per-block loops carry running addresses
     // (stage base, barrier, image row, descriptors) instead of recomputing them.
-    if (warp == 0) {
-        // ------------------------------------------------ producer: step 1, kept blocks only
+    if (warp == 0 || warp == 2 + kEpi) {
+        // ------------------------------------------------ producers: step 1, kept blocks only
+        // Issuing a tiled copy costs the issuing thread 90 to 170 cycles and every pass of its loop some 170 more
+        // (measured with cycle stamps: wait 55, byte count 20, copy 155, loop 170), so one thread that brings
+        // both operands fills a stage about every 450 cycles.  Two threads share the work by operand: warp 0
+        // brings the weight tiles and posts the byte count of the whole stage (the only arrival the `full` barrier
+        // expects), the warp after the epilogue warps walks the block columns and brings the X tiles.  Both wait
+        // for the same `empty` phase, so neither writes a stage that is still being read; bytes of X that land
+        // before the count is posted are carried by the barrier's transaction count until the arrival comes.
         if (lane == 0) {
-            constexpr int kAhead = 8;            // block columns held in registers ahead of their use
             const uint32_t ring_end = ring + p.num_stages * p.stage_bytes;
             const uint32_t entry_rows = p.entry_bytes >> 8;      // image rows (256 bytes) per walk entry
-            const bool tiled = p.a_map && p.x_map_3d;
             uint32_t dst = ring, full = bar_full, empty = bar_empty, ph = 0;
-            int fill_no = 0;
-            for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
-                const int st = t % p.nst, ct = t / p.nst;
-                const int len = walk_len[st];
-                const int32_t *cols = walk_col + (int64_t)st * p.wcap;
-                const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
-                const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
-                int arow0 = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
-                // The block column of entry e is a load in this thread's serial loop; left where it is used
-                // it costs a round trip per stage.  Keep the next kAhead in registers.
-                bool ok = true;
-              for (int q = 0; q < p.stack && ok; ++q) {
-                int arow = arow0 + q * p.wcap * (int)entry_rows;      // image copy q (stack > 1 only with one CTA tile)
-                const int xbox = (ct * p.stack + q) * NT;             // first 64-column box of this group's X columns
-                int col_q[kAhead];
+            int fill_no = 0;     // test hook: fill number p.skip_fill gets no copies, so its `full` barrier never
+                                 // completes and the bounded wait of the MMA issuer ends the kernel with CRISP_TIMEOUT
+            if (warp == 0) {
+                for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                    const int st = t % p.nst;
+                    const int len = walk_len[st];
+                    const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
+                    const int arow0 = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
+                    bool ok = true;
+                    for (int q = 0; q < p.stack && ok; ++q) {             // image copy q (stack > 1 only with one CTA tile)
+                        int arow = arow0 + q * p.wcap * (int)entry_rows;
+                        const uint8_t *src = img + (int64_t)q * p.wcap * p.entry_bytes;
+                        for (int e = 0; e < len; ++e) {
+                            if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
+                            mbar_expect_tx(full, tx_bytes);
+                            if (fill_no++ != p.skip_fill) {
+                                // the weight tile comes in as a box of 256-byte image rows (tiled copies pipeline,
+                                // untiled bulk copies are served one at a time)
+                                if (p.a_map) tma_load_2d(dst, &map_a, 0, arow, full);
+                                else bulk_load(dst, src, p.entry_bytes, full);
+                            }
+                            arow += (int)entry_rows; src += p.entry_bytes;
+                            dst += p.stage_bytes; full += 8; empty += 8;
+                            if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
+                        }
+                    }
+                    if (!ok) break;
+                }
+            } else {
+                constexpr int kAhead = 8;            // block columns held in registers ahead of their use
+                dst += p.entry_bytes;
+                for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                    const int st = t % p.nst, ct = t / p.nst;
+                    const int len = walk_len[st];
+                    const int32_t *cols = walk_col + (int64_t)st * p.wcap;
+                    const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
+                    // The block column of entry e is a load in this thread's serial loop; left where it is used
+                    // it costs a round trip per stage.  Keep the next kAhead in registers.
+                    bool ok = true;
+                    for (int q = 0; q < p.stack && ok; ++q) {
+                        const int xbox = (ct * p.stack + q) * NT;         // first 64-column box of this group's X columns
+                        int col_q[kAhead];
 #pragma unroll
-                for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
-                for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
+                        for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
+                        for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
 #pragma unroll
-                    for (int u = 0; u < kAhead; ++u) {
-                        const int e = e0 + u;
-                        if (e >= len) break;
-                        const int jb = col_q[u];
-                        const int krow = jb * p.bk;
-                        if (e + kAhead < len) col_q[u] = cols[e + kAhead];
-                        if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
-                        mbar_expect_tx(full, tx_bytes);
-                        if (fill_no++ == p.skip_fill) {
-                            // test hook: this fill's copies are left out, so its `full` barrier never completes
-                            // and the bounded wait of the MMA issuer must end the kernel with CRISP_TIMEOUT
-                            if constexpr (kConv) arow += (int)entry_rows; else if (tiled) arow += (int)entry_rows;
-                        } else
-                        if constexpr (kConv) {
-                            // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box shifted
-                            // by the tap; pixels outside the image read as zero (the convolution's padding)
-                            const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
-                            const int ti = tap / p.cv_kw, tj = tap - ti * p.cv_kw;
-                            tma_load_2d(dst, &map_a, 0, arow, full);
-                            tma_load_4d(dst + p.entry_bytes, &map_x, c0, org.x + tj - p.cv_pad, org.y + ti - p.cv_pad, org.b, full);
-                            arow += (int)entry_rows;
-                        } else if (tiled) {
-                            // tiled loads pipeline (untiled bulk copies are served one at a time): the weight
-                            // tile comes in as a box of 256-byte image rows, the NT boxes of X as one 3-D load
-                            tma_load_2d(dst, &map_a, 0, arow, full);
-                            tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, xbox, full);
-                            arow += (int)entry_rows;
-                        } else {
-                            if (p.a_map)
-                                tma_load_2d(dst, &map_a, 0, arow + e * (int)entry_rows, full);
-                            else
-                                bulk_load(dst, img + ((int64_t)q * p.wcap + e) * p.entry_bytes, p.entry_bytes, full);
-                            if (p.x_map_3d) {
-                                tma_load_3d(dst + p.entry_bytes, &map_x, 0, krow, xbox, full);
-                            } else {
+                            for (int u = 0; u < kAhead; ++u) {
+                                const int e = e0 + u;
+                                if (e >= len) break;
+                                const int jb = col_q[u];
+                                const int krow = jb * p.bk;
+                                if (e + kAhead < len) col_q[u] = cols[e + kAhead];
+                                if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
+                                if (fill_no++ != p.skip_fill) {
+                                    if constexpr (kConv) {
+                                        // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box
+                                        // shifted by the tap; pixels outside the image read as zero (the padding)
+                                        const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
+                                        const int ti = tap / p.cv_kw, tj = tap - ti * p.cv_kw;
+                                        tma_load_4d(dst, &map_x, c0, org.x + tj - p.cv_pad, org.y + ti - p.cv_pad, org.b, full);
+                                    } else if (p.x_map_3d) {
+                                        tma_load_3d(dst, &map_x, 0, krow, xbox, full);       // the NT boxes of X as one copy
+                                    } else {
 #pragma unroll
-                                for (int b = 0; b < NT; ++b)
-                                    tma_load_2d(dst + p.entry_bytes + b * p.box_bytes, &map_x, (xbox + b) * kBoxN, krow, full);
+                                        for (int b = 0; b < NT; ++b)
+                                            tma_load_2d(dst + b * p.box_bytes, &map_x, (xbox + b) * kBoxN, krow, full);
+                                    }
+                                }
+                                dst += p.stage_bytes; full += 8; empty += 8;
+                                if (dst == ring_end + p.entry_bytes) { dst = ring + p.entry_bytes; full = bar_full; empty = bar_empty; ph ^= 1u; }
                             }
                         }
-                        dst += p.stage_bytes; full += 8; empty += 8;
-                        if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
                     }
+                    if (!ok) break;
                 }
-              }
-                if (!ok) break;
             }
         }
     } else if (warp == 1) {
@@ -482,7 +503,7 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
             }
         }
-    } else {
+    } else if (warp < 2 + kEpi) {
         // ------------------------------------------------ epilogue: TMEM -> registers -> smem -> TMA store
         // Warp w may touch TMEM lanes 32*(w%4)..; the kEpi/4 warps that share a lane quarter split the
         // tile's columns among them when the shares are whole 64-column boxes: a warp first pulls its
@@ -767,7 +788,7 @@ struct TcVariant {
 template <int NT, bool kSparse, int kAccStages, typename OutT, int kEpi, bool kConv>
 TcVariant make_variant() {
     static std::atomic<size_t> configured[kMaxDevices];
-    return TcVariant{spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi, kConv>, 64 + 32 * kEpi, configured};
+    return TcVariant{spmm_tc_kernel<NT, kSparse, kAccStages, OutT, kEpi, kConv>, 96 + 32 * kEpi, configured};
 }
 
 cudaError_t prepare_variant(const TcVariant &v, int device, size_t smem) {
@@ -1152,7 +1173,7 @@ cudaError_t make_plan(const crisp_handle_s *h, int kind, const uint16_t *d_x, in
     info.tile_cols = nt * kBoxN;
     info.accumulators = acc;
     info.stack = stack;
-    info.epilogue_warps = plan->variant.threads / 32 - 2;
+    info.epilogue_warps = plan->variant.threads / 32 - 3;
     info.stages = (int)stages;
     info.ctas = plan->grid;
     info.conv = conv ? 1 : 0;
