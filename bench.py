@@ -256,7 +256,7 @@ def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=50):
     Cold L2: `iters` launches, each after an L2 flush, each in its own event pair (median and minimum).
     Warm L2: the same launch repeated back to back on the same buffers, `iters` launches in five event pairs
     (median and minimum of the five averages); for layers larger than L2 that is simply a pipelined stream of
-    launches."""
+    launches.  (measure_cells_graph adds a third protocol to the same records.)"""
     out = []
     stream = torch.cuda.current_stream()
 
@@ -310,7 +310,7 @@ def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=50):
                "ncols": layer.ncols, "nm": f"{layer.n}:{layer.m}", "block": [layer.block_rows, layer.block_k],
                "keep": round(layer.keep_ratio, 4), "kkeep": L.kkeep, "kernel": B.PATH_NAMES[launched["path"]],
                "tile_cols": launched["tile_cols"], "accumulators": launched["accumulators"],
-               "stack": launched["stack"],
+               "stack": launched["stack"], "stage_blocks": launched["stage_blocks"],
                "spmm_us": c_med, "spmm_us_min": c_min, "spmm_warm_us": w_med, "spmm_warm_us_min": w_min,
                "dense_cublas_us": dc_med, "dense_cublas_us_min": dc_min, "dense_cublas_warm_us": dw_med,
                "speedup_vs_dense_cublas": dc_med / c_med, "speedup_warm": dw_med / w_med,
@@ -330,6 +330,60 @@ def measure_cells(torch, B, dev, peaks, flush_l2, shared, iters=50):
         if layer.config != 5:
             del d_x, d_w, d_s
     return out
+
+
+def measure_cells_graph(torch, B, dev, shared, cells):
+    """Graph replay of every cell, added to the records of measure_cells: 20 launches captured in a CUDA graph and
+    replayed (median and minimum per launch over 9 replays), ours and the dense cuBLAS GEMM: device time without
+    the host's launch path and without the 2 us tick of the event timer, which is what separates layers of a few
+    microseconds; operands stay in L2 where they fit.  A pass of its own, after every other figure of the run
+    has been taken: the replays keep the GPU under load for seconds, and cold launches measured in between came
+    out up to 20 % slower (ours and cuBLAS alike)."""
+    side = torch.cuda.Stream()
+
+    def replay(fn, n=20, reps=9):
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            fn(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(n):
+                    fn(side)
+            g.replay()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(side); g.replay(); b.record(side)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3 / n)
+        del g
+        return float(np.median(ts)), float(np.min(ts))
+
+    for rec, layer in zip(cells, all_cells()):
+        if layer.config == 5:
+            d_s, d_w, d_x = shared
+        else:
+            w = wl.make_weight(layer)
+            d_s = torch.from_numpy(wl.make_saliency(layer, w)).to(dev)
+            d_w = torch.from_numpy(w.view(np.int16)).to(dev).view(torch.bfloat16)
+            d_x = device_activation(torch, layer, dev)
+        d_y = torch.empty((layer.rows, layer.ncols), dtype=torch.bfloat16, device=dev)
+        L = B.HybridLayer(layer.rows, layer.k, layer.n, layer.m, layer.block_rows, layer.block_k,
+                          layer.keep_ratio, device=dev)
+        L.build_mask(d_s).encode(d_w)
+        g_med, g_min = replay(lambda st: L.spmm(d_x, y=d_y, stream=st))
+        dg_med, dg_min = replay(lambda st: torch.matmul(d_w, d_x, out=d_y))
+        rec.update({"spmm_graph_us": g_med, "spmm_graph_us_min": g_min, "dense_cublas_graph_us": dg_med,
+                    "dense_cublas_graph_us_min": dg_min, "speedup_graph": dg_med / g_med})
+        if L.device_status() != 0:
+            rec["device_status"] = L.device_status()
+        L.close()
+        del d_y
+        if layer.config != 5:
+            del d_x, d_w, d_s
+    return cells
 
 
 def measure_two_addends(torch, B, dev, peaks, flush_l2, shared, iters=30):
@@ -380,9 +434,12 @@ def summarise_cells(cells):
         if not cs:
             continue
         ours, dense = sum(c["spmm_us"] for c in cs), sum(c["dense_cublas_us"] for c in cs)
+        g_ours, g_dense = sum(c["spmm_graph_us"] for c in cs), sum(c["dense_cublas_graph_us"] for c in cs)
         fr = [c["roofline_frac"] for c in cs]
         out[name] = {"layers": len(cs), "spmm_us_sum": ours, "dense_cublas_us_sum": dense,
                      "speedup_vs_dense_cublas": dense / ours,
+                     "spmm_graph_us_sum": g_ours, "dense_cublas_graph_us_sum": g_dense, "speedup_graph": g_dense / g_ours,
+                     "faster_than_dense_graph": sum(1 for c in cs if c["speedup_graph"] >= 1.0),
                      "useful_tflops": sum(c["useful_tflops"] * c["spmm_us"] for c in cs) / ours,
                      "roofline_frac_min": min(fr), "roofline_frac_median": float(np.median(fr)),
                      "roofline_frac_max": max(fr),
@@ -888,13 +945,14 @@ def run_ours(args, layer, rank, world):
 
     if rank == 0 and world == 1 and not args.no_cells and args.workload.startswith("sweep_"):
         cells = measure_cells(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x), iters=args.cell_iters)
-        out["summary"] = summarise_cells(cells)
         out["cells"] = cells
         out["global_rank"] = measure_global_rank(torch, B, dev, not args.no_cpu_baseline)
         out["conv"] = measure_conv(torch, B, dev, peaks, flush_l2)
         out["saliency"] = measure_saliency(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
         out["pruning_iteration"] = measure_iteration(torch, B, dev, not args.no_cpu_baseline)
         out["two_addend_form"] = measure_two_addends(torch, B, dev, peaks, flush_l2, (d_s, d_w, d_x))
+        measure_cells_graph(torch, B, dev, (d_s, d_w, d_x), cells)
+        out["summary"] = summarise_cells(cells)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         cols = oracle_sample_cols(layer, w, s, x)
@@ -934,25 +992,31 @@ def render_markdown(d):
     def row(x):
         fr = "-" if x["roofline_frac"] is None else f"{x['roofline_frac']:.2f} / {x['roofline_frac_literal']:.2f}"
         return (f"| {x['workload']} | {x['rows']}x{x['k']}x{x['ncols']} | {x['nm']} | {x['kkeep']} | {x['kernel'].replace('_tcgen05', '')} "
-                f"{x['tile_cols']}c/{x['accumulators']}a{'/s' + str(x['stack']) if x['stack'] > 1 else ''} | {x['spmm_us']:.1f} ({x['spmm_us_min']:.1f}) | "
+                f"{x['tile_cols']}c/{x['accumulators']}a{'/s' + str(x['stack']) if x['stack'] > 1 else ''}"
+                f"{'/b' + str(x['stage_blocks']) if x.get('stage_blocks', 1) > 1 else ''} | {x['spmm_us']:.1f} ({x['spmm_us_min']:.1f}) | "
                 f"{x['spmm_warm_us']:.1f} | {x['dense_cublas_us']:.1f} | {x['speedup_vs_dense_cublas']:.2f} | "
+                f"{x['spmm_graph_us']:.2f} | {x['dense_cublas_graph_us']:.2f} | {x['speedup_graph']:.2f} | "
                 f"{x['useful_tflops']:.1f} | {fr} |")
 
-    head = ("| workload | rows x k x ncols | N:M | kkeep | kernel (tile columns / accumulators) | SpMM us cold: median (min) | warm | "
-            "dense cuBLAS us | x dense | useful TFLOP/s | roofline slot-aware / literal |\n|---|---|---|---|---|---|---|---|---|---|---|")
+    head = ("| workload | rows x k x ncols | N:M | kkeep | kernel (tile columns / accumulators / stack / blocks per stage) | "
+            "SpMM us cold: median (min) | warm | dense cuBLAS us | x dense | graph replay us | dense cuBLAS graph us | x dense (graph) | "
+            "useful TFLOP/s | roofline slot-aware / literal |\n|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for cfg, title in ((5, "Sweep (config 5) and 3:4"), (1, "Config 1"), (2, "Config 2"), (3, "Config 3: VGG-16 stand-in"),
                        (4, "Config 4: MobileNetV2 stand-in")):
         rows = [x for x in cells if x["config"] == cfg]
         if rows:
             o.append(f"\n**{title}** (`cells`)\n\n" + head + "\n" + "\n".join(row(x) for x in rows))
     if "summary" in d:
-        o.append("\n**Per family** (`summary`; layers without a kept block left out)\n\n| family | layers | ours us | dense cuBLAS us | x dense | "
-                 "useful TFLOP/s | roofline min / median / max | faster than dense |\n|---|---|---|---|---|---|---|---|")
+        o.append("\n**Per family** (`summary`; layers without a kept block left out; cold = each launch after an L2 flush in its own "
+                 "event pair, graph = replay of 20 captured launches)\n\n| family | layers | ours us (cold) | dense cuBLAS us | x dense | "
+                 "ours us (graph) | dense cuBLAS us (graph) | x dense (graph) | useful TFLOP/s | roofline min / median / max | "
+                 "faster than dense cold / graph |\n|---|---|---|---|---|---|---|---|---|---|---|")
         for k, v in d["summary"].items():
             if "spmm_us_sum" in v:
                 o.append(f"| {k} | {v['layers']} | {v['spmm_us_sum']:.1f} | {v['dense_cublas_us_sum']:.1f} | {v['speedup_vs_dense_cublas']:.2f} | "
+                         f"{v['spmm_graph_us_sum']:.1f} | {v['dense_cublas_graph_us_sum']:.1f} | {v['speedup_graph']:.2f} | "
                          f"{v['useful_tflops']:.1f} | {v['roofline_frac_min']:.2f} / {v['roofline_frac_median']:.2f} / {v['roofline_frac_max']:.2f} | "
-                         f"{v['faster_than_dense']} of {v['layers']} |")
+                         f"{v['faster_than_dense']} / {v['faster_than_dense_graph']} of {v['layers']} |")
         lo = d["summary"]["sweep_keep_le_0.5"]
         o.append(f"\nSweep cells with keep <= 0.5: {lo['at_or_above_60pct_of_roofline']} of {lo['cells']} at or above 0.60 of the "
                  f"slot-aware roofline, {lo['faster_than_dense']} of {lo['cells']} faster than dense cuBLAS.")

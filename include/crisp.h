@@ -113,6 +113,7 @@ typedef struct {
     int32_t stages;           /* depth of the shared-memory ring                                 */
     int32_t ctas;             /* grid size                                                       */
     int32_t conv;             /* 1 if the activations were gathered from an NHWC tensor          */
+    int32_t stage_blocks;     /* kept blocks per pipeline stage (1, 2 or 4)                      */
 } crisp_launch_info_t;
 
 /* kkeep = floor(keep_ratio * nblk + 0.5), clamped to [0, nblk], evaluated in double on the
@@ -405,6 +406,12 @@ CRISP_API crisp_status_t crisp_last_launch(crisp_handle_t h, crisp_launch_info_t
  * The paper has no counterpart; Sec. III-E's pipeline has no failure model. */
 CRISP_API crisp_status_t crisp_set_tuning(crisp_handle_t h, int32_t tile_boxes, uint64_t wait_limit_cycles,
                                           int32_t skip_fill);
+
+/* Upper bound on the kept blocks that one pipeline stage of the tensor-core kernels takes (1, 2 or 4;
+ * 0 = chosen by the library, the default).  A stage of several blocks shares one wait, one weight-tile copy
+ * and one commit among them; results do not depend on it.  Takes effect at the next product.
+ * The paper has no counterpart (Sec. III-E names no pipeline depth).  Error: INVALID_ARG. */
+CRISP_API crisp_status_t crisp_set_stage_blocks(crisp_handle_t h, int32_t max_blocks);
 
 /* Clear the device status word of the handle on `stream` (after a reported CRISP_TIMEOUT). */
 CRISP_API crisp_status_t crisp_reset_status(crisp_handle_t h, void *stream);

@@ -36,7 +36,8 @@ class ConvDesc(C.Structure):
 
 class LaunchInfo(C.Structure):
     _fields_ = [("path", C.c_int32), ("tile_cols", C.c_int32), ("accumulators", C.c_int32), ("stack", C.c_int32),
-                ("epilogue_warps", C.c_int32), ("stages", C.c_int32), ("ctas", C.c_int32), ("conv", C.c_int32)]
+                ("epilogue_warps", C.c_int32), ("stages", C.c_int32), ("ctas", C.c_int32), ("conv", C.c_int32),
+                ("stage_blocks", C.c_int32)]
 
     def as_dict(self):
         return {f: int(getattr(self, f)) for f, _ in self._fields_}
@@ -100,6 +101,7 @@ def load(path: Optional[str] = None):
         "crisp_device_status": [vp, vp, P(i32)],
         "crisp_last_launch": [vp, P(LaunchInfo)],
         "crisp_set_tuning": [vp, i32, C.c_uint64, i32],
+        "crisp_set_stage_blocks": [vp, i32],
         "crisp_reset_status": [vp, vp],
         "crisp_bytes_model": [vp, i64, i32, P(BytesModel)],
         "crisp_mask_scores": [P(LayerDesc), vp, P(vp), P(vp)],
@@ -334,6 +336,11 @@ def crisp_set_tuning(handle: int, tile_boxes: int = 0, wait_limit_cycles: int = 
     _check(load().crisp_set_tuning(handle, tile_boxes, wait_limit_cycles, skip_fill), "crisp_set_tuning")
 
 
+def crisp_set_stage_blocks(handle: int, max_blocks: int = 0):
+    """Most kept blocks one pipeline stage may take (1, 2, 4; 0 = chosen by the library)."""
+    _check(load().crisp_set_stage_blocks(handle, max_blocks), "crisp_set_stage_blocks")
+
+
 def crisp_reset_status(handle: int, stream=None):
     _check(load().crisp_reset_status(handle, _stream(stream)), "crisp_reset_status")
 
@@ -494,6 +501,10 @@ class HybridLayer:
 
     def set_tuning(self, tile_boxes=0, wait_limit_cycles=0, skip_fill=-1):
         crisp_set_tuning(self.handle, tile_boxes, wait_limit_cycles, skip_fill)
+        return self
+
+    def set_stage_blocks(self, max_blocks=0):
+        crisp_set_stage_blocks(self.handle, max_blocks)
         return self
 
     def reset_status(self, stream=None):

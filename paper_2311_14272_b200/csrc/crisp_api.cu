@@ -214,10 +214,11 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     h->epilogue = crisp::Epilogue{nullptr, 0};
     const char *nt_env = std::getenv("CRISP_TC_NT");          // 64-column boxes per CTA tile, tuning only; read once
     h->nt_override = nt_env ? std::atoi(nt_env) : 0;
+    h->group_override = 0;
     h->wait_limit_cycles = 0;
     h->debug_skip_stage = -1;
     h->plan = nullptr;
-    h->last = crisp_launch_info_t{-1, 0, 0, 1, 0, 0, 0, 0};
+    h->last = crisp_launch_info_t{-1, 0, 0, 1, 0, 0, 0, 0, 1};
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
     // 128-row blocks: one kept block is one tensor-core tile, so the encode kernel writes it directly
@@ -339,6 +340,12 @@ crisp_status_t crisp_spmm_conv(crisp_handle_t h, const uint16_t *d_act_nhwc, con
 crisp_status_t crisp_last_launch(crisp_handle_t h, crisp_launch_info_t *out) {
     if (!h || !out) return CRISP_INVALID_ARG;
     *out = h->last;
+    return CRISP_OK;
+}
+
+crisp_status_t crisp_set_stage_blocks(crisp_handle_t h, int32_t max_blocks) {
+    if (!h || (max_blocks != 0 && max_blocks != 1 && max_blocks != 2 && max_blocks != 4)) return CRISP_INVALID_ARG;
+    h->group_override = max_blocks;
     return CRISP_OK;
 }
 

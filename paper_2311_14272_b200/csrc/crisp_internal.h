@@ -65,6 +65,7 @@ struct crisp_handle_s {
     int forced_path;        // -1 = default
     crisp::Epilogue epilogue;
     int nt_override;        // tuning: 64-column boxes per CTA tile (0 = chosen by the library)
+    int group_override;     // tuning: most kept blocks a pipeline stage may take (0 = chosen by the library)
     unsigned long long wait_limit_cycles;   // bound of every in-kernel wait (0 = default)
     int debug_skip_stage;   // test hook: the producer leaves out the loads of this pipeline fill (-1 = none)
     crisp::TcPlan *plan;    // cached launch plan of the last tensor-core product (or nullptr)

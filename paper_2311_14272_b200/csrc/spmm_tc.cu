@@ -38,6 +38,7 @@ struct TcParams {
     int nst, wcap, bk, n_col_tiles, num_tiles, rows;
     int64_t ncols;
     uint32_t a_bytes, entry_bytes, box_bytes, stage_bytes, num_stages;
+    uint32_t group;             // kept blocks per pipeline stage (1, 2 or 4): [group weight tiles + metadata | group X tiles]
     uint32_t addends;           // sparse tiles (each a_bytes + metadata) per walk entry: 2 when a block with up to four
                                 // values per aligned 4-group is multiplied as two 2:4-compliant addends
     uint32_t stg_bufs;          // staging tiles per epilogue warp (1, 2 or 4): stores in flight per warp
@@ -270,48 +271,103 @@ __device__ __forceinline__ void mma_role(const TcParams &p, const MmaRoleArgs &a
     // contiguous (K-major operand, 128-byte rows in 1024-byte groups of 8, a K step is 64 or 32 bytes)
     constexpr uint32_t idesc = kConv ? (make_idesc(kTileN, kSparse) & ~(1u << 16)) : make_idesc(kTileN, kSparse);
     const uint64_t a_desc0 = make_smem_desc(a.ring, 2048, 128, kLayoutNone);
-    const uint64_t b_desc0 = kConv ? make_smem_desc(a.ring + p.entry_bytes, 16, 1024, kLayoutSw128)
-                                   : make_smem_desc(a.ring + p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
+    const uint64_t b_desc0 = kConv ? make_smem_desc(a.ring + p.group * p.entry_bytes, 16, 1024, kLayoutSw128)
+                                   : make_smem_desc(a.ring + p.group * p.entry_bytes, p.box_bytes, 1024, kLayoutSw128);
     constexpr uint32_t b_step = kConv ? (kSparse ? 4u : 2u) : (kSparse ? 256u : 128u);
     const uint64_t m_desc0 = make_smem_desc(a.ring + p.a_bytes, 128, 128, kLayoutNone);
     const uint32_t stage_step = p.stage_bytes >> 4, ring_span = p.num_stages * stage_step;
+    const uint32_t a_step = p.entry_bytes >> 4, x_step = ((uint32_t)(kTileN / kBoxN) * p.box_bytes) >> 4;   // per block of a stage
+    const int group = (int)p.group;
     uint32_t off = 0, full = a.bar_full, empty = a.bar_empty, ph = 0, acc = 0, acc_ph = 0, meta_buf = 0;
+    if (group == 1) {
+        // one kept block per stage: the plain loop (large tiles; every extra instruction here costs the headline cells)
+        for (int t = blockIdx.x; t < p.num_tiles && !*a.abort_flag; t += gridDim.x) {
+            const int len = min(a.walk_len[t % p.nst], p.wcap) * p.stack;
+            if (!mbar_wait(a.bar_tempty + 8 * acc, acc_ph ^ 1u, a.abort_flag, p.wait_limit)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = a.tmem_base + acc * kTileN;
+            uint32_t accum = 0;
+            bool ok = true;
+            for (int e = 0; e < len; ++e) {
+                if (!mbar_wait(full, ph, a.abort_flag, p.wait_limit)) { ok = false; break; }
+                tc_fence_after();
+                const uint64_t ad = a_desc0 + off, bd = b_desc0 + off;
+                if constexpr (kSparse) {
+                    const uint32_t meta_tmem = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                    tmem_copy_128x128b(meta_tmem, m_desc0 + off);
+#pragma unroll
+                    for (int j = 0; j < NM; ++j)
+                        mma_sparse(d_tmem, ad + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), accum | (uint32_t)j,
+                                   meta_tmem + (j & ~1));
+                    meta_buf ^= 1u;
+                    if (p.addends == 2) {               // second addend of the block: same X tile, same accumulator
+                        const uint32_t sub = (p.a_bytes + kMetaBytes) >> 4;
+                        const uint32_t meta2 = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                        tmem_copy_128x128b(meta2, m_desc0 + off + sub);
+#pragma unroll
+                        for (int j = 0; j < NM; ++j)
+                            mma_sparse(d_tmem, ad + sub + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), 1u, meta2 + (j & ~1));
+                        meta_buf ^= 1u;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * b_step, idesc, accum | (uint32_t)j);
+                }
+                accum = 1u;
+                mma_commit(empty);                      // stage reusable once these MMAs have read it
+                off += stage_step; full += 8; empty += 8;
+                if (off == ring_span) { off = 0; full = a.bar_full; empty = a.bar_empty; ph ^= 1u; }
+            }
+            if (!ok) break;
+            mma_commit(a.bar_tfull + 8 * acc);          // accumulator complete
+            if (++acc == kAccStages) { acc = 0; acc_ph ^= 1u; }
+        }
+        return;
+    }
     for (int t = blockIdx.x; t < p.num_tiles && !*a.abort_flag; t += gridDim.x) {
-        const int len = a.walk_len[t % p.nst] * p.stack;
+        const int len = min(a.walk_len[t % p.nst], p.wcap);    // (the clamp keeps a list that was overwritten in bounds)
         if (!mbar_wait(a.bar_tempty + 8 * acc, acc_ph ^ 1u, a.abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t d_tmem = a.tmem_base + acc * kTileN;
         uint32_t accum = 0;
         bool ok = true;
-        for (int e = 0; e < len; ++e) {
-            if (!mbar_wait(full, ph, a.abort_flag, p.wait_limit)) { ok = false; break; }
-            tc_fence_after();
-            const uint64_t ad = a_desc0 + off, bd = b_desc0 + off;
-            if constexpr (kSparse) {
-                const uint32_t meta_tmem = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
-                tmem_copy_128x128b(meta_tmem, m_desc0 + off);
+        // a stacked tile walks its list once per lane group; a stage never spans two walks
+        for (int q = 0; q < p.stack && ok; ++q) {
+            for (int e = 0; e < len; e += group) {
+                if (!mbar_wait(full, ph, a.abort_flag, p.wait_limit)) { ok = false; break; }
+                tc_fence_after();
+                const int cnt = min(group, len - e);
 #pragma unroll
-                for (int j = 0; j < NM; ++j)
-                    mma_sparse(d_tmem, ad + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), accum | (uint32_t)j,
-                               meta_tmem + (j & ~1));
-                meta_buf ^= 1u;
-                if (p.addends == 2) {               // second addend of the block: same X tile, same accumulator
-                    const uint32_t sub = (p.a_bytes + kMetaBytes) >> 4;
-                    const uint32_t meta2 = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
-                    tmem_copy_128x128b(meta2, m_desc0 + off + sub);
+                for (int g = 0; g < 4; ++g) {
+                    if (g >= cnt) break;
+                    const uint64_t ad = a_desc0 + off + g * a_step, bd = b_desc0 + off + g * x_step;
+                    if constexpr (kSparse) {
+                        const uint32_t meta_tmem = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                        tmem_copy_128x128b(meta_tmem, m_desc0 + off + g * a_step);
 #pragma unroll
-                    for (int j = 0; j < NM; ++j)
-                        mma_sparse(d_tmem, ad + sub + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), 1u, meta2 + (j & ~1));
-                    meta_buf ^= 1u;
+                        for (int j = 0; j < NM; ++j)
+                            mma_sparse(d_tmem, ad + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), accum | (uint32_t)j,
+                                       meta_tmem + (j & ~1));
+                        meta_buf ^= 1u;
+                        if (p.addends == 2) {               // second addend of the block: same X tile, same accumulator
+                            const uint32_t sub = (p.a_bytes + kMetaBytes) >> 4;
+                            const uint32_t meta2 = a.tmem_base + kAccStages * kTileN + 4 * meta_buf;
+                            tmem_copy_128x128b(meta2, m_desc0 + off + g * a_step + sub);
+#pragma unroll
+                            for (int j = 0; j < NM; ++j)
+                                mma_sparse(d_tmem, ad + sub + j * 256, bd + j * b_step, idesc | (uint32_t)(j & 1), 1u, meta2 + (j & ~1));
+                            meta_buf ^= 1u;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * b_step, idesc, accum | (uint32_t)j);
+                    }
+                    accum = 1u;
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < NM; ++j) mma_dense(d_tmem, ad + j * 256, bd + j * b_step, idesc, accum | (uint32_t)j);
+                mma_commit(empty);                      // stage reusable once these MMAs have read it
+                off += stage_step; full += 8; empty += 8;
+                if (off == ring_span) { off = 0; full = a.bar_full; empty = a.bar_empty; ph ^= 1u; }
             }
-            accum = 1u;
-            mma_commit(empty);                      // stage reusable once these MMAs have read it
-            off += stage_step; full += 8; empty += 8;
-            if (off == ring_span) { off = 0; full = a.bar_full; empty = a.bar_empty; ph ^= 1u; }
         }
         if (!ok) break;
         mma_commit(a.bar_tfull + 8 * acc);          // accumulator complete
@@ -387,7 +443,8 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
-    const uint32_t tx_bytes = p.entry_bytes + NT * p.box_bytes;
+    const uint32_t x_blk_bytes = NT * p.box_bytes;           // X tile of one kept block
+    const uint32_t tx_bytes = p.entry_bytes + x_blk_bytes;   // a stage of one block
 
     // Both single-thread roles below are bound by their own dependent-instruction latency (one warp per
     // scheduler, ~5 cycles per dependent instruction), so their per-block loops carry running addresses
@@ -408,77 +465,162 @@ spmm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             int fill_no = 0;     // test hook: fill number p.skip_fill gets no copies, so its `full` barrier never
                                  // completes and the bounded wait of the MMA issuer ends the kernel with CRISP_TIMEOUT
             if (warp == 0) {
-                for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
-                    const int st = t % p.nst;
-                    const int len = walk_len[st];
-                    const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
-                    const int arow0 = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
-                    bool ok = true;
-                    for (int q = 0; q < p.stack && ok; ++q) {             // image copy q (stack > 1 only with one CTA tile)
-                        int arow = arow0 + q * p.wcap * (int)entry_rows;
-                        const uint8_t *src = img + (int64_t)q * p.wcap * p.entry_bytes;
-                        for (int e = 0; e < len; ++e) {
-                            if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
-                            mbar_expect_tx(full, tx_bytes);
-                            if (fill_no++ != p.skip_fill) {
-                                // the weight tile comes in as a box of 256-byte image rows (tiled copies pipeline,
-                                // untiled bulk copies are served one at a time)
-                                if (p.a_map) tma_load_2d(dst, &map_a, 0, arow, full);
-                                else bulk_load(dst, src, p.entry_bytes, full);
+                if (p.group == 1) {       // one kept block per stage: the plain loop
+                    for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                        const int st = t % p.nst;
+                        const int len = min(walk_len[st], p.wcap);
+                        const uint8_t *img = p.image + (int64_t)st * p.wcap * p.entry_bytes;
+                        const int arow0 = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
+                        bool ok = true;
+                        for (int q = 0; q < p.stack && ok; ++q) {             // image copy q (stack > 1 only with one CTA tile)
+                            int arow = arow0 + q * p.wcap * (int)entry_rows;
+                            const uint8_t *src = img + (int64_t)q * p.wcap * p.entry_bytes;
+                            for (int e = 0; e < len; ++e) {
+                                if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
+                                mbar_expect_tx(full, tx_bytes);
+                                if (fill_no++ != p.skip_fill) {
+                                    // the weight tile comes in as a box of 256-byte image rows (tiled copies pipeline,
+                                    // untiled bulk copies are served one at a time)
+                                    if (p.a_map) tma_load_2d(dst, &map_a, 0, arow, full);
+                                    else bulk_load(dst, src, p.entry_bytes, full);
+                                }
+                                arow += (int)entry_rows; src += p.entry_bytes;
+                                dst += p.stage_bytes; full += 8; empty += 8;
+                                if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
                             }
-                            arow += (int)entry_rows; src += p.entry_bytes;
-                            dst += p.stage_bytes; full += 8; empty += 8;
-                            if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
                         }
+                        if (!ok) break;
                     }
-                    if (!ok) break;
+                } else {
+                    for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                        const int st = t % p.nst;
+                        const int len = min(walk_len[st], p.wcap);
+                        const int arow0 = (int)(((int64_t)st * p.wcap * p.entry_bytes) >> 8);
+                        bool ok = true;
+                        for (int q = 0; q < p.stack && ok; ++q) {             // image copy q (stack > 1 only with one CTA tile)
+                            int arow = arow0 + q * p.wcap * (int)entry_rows;
+                            for (int e = 0; e < len; e += (int)p.group) {
+                                if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
+                                // A stage holds `group` consecutive walk entries.  Their weight tiles are one box of the
+                                // image (a whole box also where the walk ends inside it: the rows beyond are the next
+                                // entries of the image or, past its end, zero fill, and no MMA reads them); X comes per block.
+                                const uint32_t cnt = (uint32_t)min((int)p.group, len - e);
+                                mbar_expect_tx(full, p.group * p.entry_bytes + cnt * x_blk_bytes);
+                                if (fill_no++ != p.skip_fill) tma_load_2d(dst, &map_a, 0, arow, full);   // (the weight map is tiled here)
+                                arow += (int)(p.group * entry_rows);
+                                dst += p.stage_bytes; full += 8; empty += 8;
+                                if (dst == ring_end) { dst = ring; full = bar_full; empty = bar_empty; ph ^= 1u; }
+                            }
+                        }
+                        if (!ok) break;
+                    }
                 }
             } else {
-                constexpr int kAhead = 8;            // block columns held in registers ahead of their use
-                dst += p.entry_bytes;
-                for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
-                    const int st = t % p.nst, ct = t / p.nst;
-                    const int len = walk_len[st];
-                    const int32_t *cols = walk_col + (int64_t)st * p.wcap;
-                    const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
-                    // The block column of entry e is a load in this thread's serial loop; left where it is used
-                    // it costs a round trip per stage.  Keep the next kAhead in registers.
-                    bool ok = true;
-                    for (int q = 0; q < p.stack && ok; ++q) {
-                        const int xbox = (ct * p.stack + q) * NT;         // first 64-column box of this group's X columns
-                        int col_q[kAhead];
+                if (p.group == 1) {       // one kept block per stage: the plain loop
+                    constexpr int kAhead = 8;            // block columns held in registers ahead of their use
+                    dst += p.entry_bytes;
+                    for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                        const int st = t % p.nst, ct = t / p.nst;
+                        const int len = min(walk_len[st], p.wcap);
+                        const int32_t *cols = walk_col + (int64_t)st * p.wcap;
+                        const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
+                        // The block column of entry e is a load in this thread's serial loop; left where it is used
+                        // it costs a round trip per stage.  Keep the next kAhead in registers.
+                        bool ok = true;
+                        for (int q = 0; q < p.stack && ok; ++q) {
+                            const int xbox = (ct * p.stack + q) * NT;         // first 64-column box of this group's X columns
+                            int col_q[kAhead];
 #pragma unroll
-                        for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
-                        for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
+                            for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
+                            for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
 #pragma unroll
-                            for (int u = 0; u < kAhead; ++u) {
-                                const int e = e0 + u;
-                                if (e >= len) break;
-                                const int jb = col_q[u];
-                                const int krow = jb * p.bk;
-                                if (e + kAhead < len) col_q[u] = cols[e + kAhead];
-                                if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
-                                if (fill_no++ != p.skip_fill) {
-                                    if constexpr (kConv) {
-                                        // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box
-                                        // shifted by the tap; pixels outside the image read as zero (the padding)
-                                        const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
-                                        const int ti = tap / p.cv_kw, tj = tap - ti * p.cv_kw;
-                                        tma_load_4d(dst, &map_x, c0, org.x + tj - p.cv_pad, org.y + ti - p.cv_pad, org.b, full);
-                                    } else if (p.x_map_3d) {
-                                        tma_load_3d(dst, &map_x, 0, krow, xbox, full);       // the NT boxes of X as one copy
-                                    } else {
+                                for (int u = 0; u < kAhead; ++u) {
+                                    const int e = e0 + u;
+                                    if (e >= len) break;
+                                    const int jb = col_q[u];
+                                    const int krow = jb * p.bk;
+                                    if (e + kAhead < len) col_q[u] = cols[e + kAhead];
+                                    if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
+                                    if (fill_no++ != p.skip_fill) {
+                                        if constexpr (kConv) {
+                                            // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box
+                                            // shifted by the tap; pixels outside the image read as zero (the padding)
+                                            const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
+                                            const int ti = tap / p.cv_kw, tj = tap - ti * p.cv_kw;
+                                            tma_load_4d(dst, &map_x, c0, org.x + tj - p.cv_pad, org.y + ti - p.cv_pad, org.b, full);
+                                        } else if (p.x_map_3d) {
+                                            tma_load_3d(dst, &map_x, 0, krow, xbox, full);       // the NT boxes of X as one copy
+                                        } else {
 #pragma unroll
-                                        for (int b = 0; b < NT; ++b)
-                                            tma_load_2d(dst + b * p.box_bytes, &map_x, (xbox + b) * kBoxN, krow, full);
+                                            for (int b = 0; b < NT; ++b)
+                                                tma_load_2d(dst + b * p.box_bytes, &map_x, (xbox + b) * kBoxN, krow, full);
+                                        }
                                     }
+                                    dst += p.stage_bytes; full += 8; empty += 8;
+                                    if (dst == ring_end + p.entry_bytes) { dst = ring + p.entry_bytes; full = bar_full; empty = bar_empty; ph ^= 1u; }
                                 }
-                                dst += p.stage_bytes; full += 8; empty += 8;
-                                if (dst == ring_end + p.entry_bytes) { dst = ring + p.entry_bytes; full = bar_full; empty = bar_empty; ph ^= 1u; }
                             }
                         }
+                        if (!ok) break;
                     }
-                    if (!ok) break;
+                } else {
+                    constexpr int kAhead = 8;            // block columns held in registers ahead of their use
+                    dst += p.group * p.entry_bytes;
+                    const int gmask = (int)p.group - 1;
+                    bool issue = true;
+                    for (int t = blockIdx.x; t < p.num_tiles && !*abort_flag; t += gridDim.x) {
+                        const int st = t % p.nst, ct = t / p.nst;
+                        const int len = min(walk_len[st], p.wcap);
+                        const int32_t *cols = walk_col + (int64_t)st * p.wcap;
+                        const TileOrigin org = tile_origin<kConv>(p, ct, kTileN);
+                        // The block column of entry e is a load in this thread's serial loop; left where it is used
+                        // it costs a round trip per stage.  Keep the next kAhead in registers.
+                        bool ok = true;
+                        for (int q = 0; q < p.stack && ok; ++q) {
+                            const int xbox = (ct * p.stack + q) * NT;         // first 64-column box of this group's X columns
+                            int col_q[kAhead];
+#pragma unroll
+                            for (int u = 0; u < kAhead; ++u) col_q[u] = u < len ? cols[u] : 0;
+                            for (int e0 = 0; e0 < len && ok; e0 += kAhead) {
+#pragma unroll
+                                for (int u = 0; u < kAhead; ++u) {
+                                    const int e = e0 + u;
+                                    if (e >= len) break;
+                                    const int jb = col_q[u];
+                                    const int krow = jb * p.bk;
+                                    if (e + kAhead < len) col_q[u] = cols[e + kAhead];
+                                    const int g = e & gmask;                  // position of the block in its stage
+                                    if (g == 0) {
+                                        if (!mbar_wait(empty, ph ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
+                                        issue = fill_no++ != p.skip_fill;
+                                    }
+                                    const uint32_t xdst = dst + (uint32_t)g * x_blk_bytes;
+                                    if (issue) {
+                                        if constexpr (kConv) {
+                                            // block jb = filter tap (i, j), channels [c0, c0 + bk): the tile's pixel box
+                                            // shifted by the tap; pixels outside the image read as zero (the padding)
+                                            const int tap = jb / p.cv_cpt, c0 = (jb - tap * p.cv_cpt) * p.bk;
+                                            const int ti = tap / p.cv_kw, tj = tap - ti * p.cv_kw;
+                                            tma_load_4d(xdst, &map_x, c0, org.x + tj - p.cv_pad, org.y + ti - p.cv_pad, org.b, full);
+                                        } else if (p.x_map_3d) {
+                                            tma_load_3d(xdst, &map_x, 0, krow, xbox, full);      // the NT boxes of X as one copy
+                                        } else {
+#pragma unroll
+                                            for (int b = 0; b < NT; ++b)
+                                                tma_load_2d(xdst + b * p.box_bytes, &map_x, (xbox + b) * kBoxN, krow, full);
+                                        }
+                                    }
+                                    if (g == gmask || e == len - 1) {         // last block of the stage
+                                        dst += p.stage_bytes; full += 8; empty += 8;
+                                        if (dst == ring_end + p.group * p.entry_bytes) {
+                                            dst = ring + p.group * p.entry_bytes; full = bar_full; empty = bar_empty; ph ^= 1u;
+                                        }
+                                    }
+                                }
+                            }
+                        }
+                        if (!ok) break;
+                    }
                 }
             }
         }
@@ -973,7 +1115,7 @@ struct TcPlan {
     // key
     const void *x, *y, *bias;
     int64_t ldx, ldy, ncols;
-    int y_dtype, relu, nt_override, device, skip_stage;
+    int y_dtype, relu, nt_override, group_override, device, skip_stage;
     unsigned long long wait_limit;
     bool has_conv;
     ConvGeom conv;
@@ -1065,7 +1207,7 @@ cudaError_t make_plan(const crisp_handle_s *h, int kind, const uint16_t *d_x, in
     p.num_tiles = (int)tiles;
     p.a_bytes = L.a_bytes; p.entry_bytes = L.entry_bytes; p.addends = (uint32_t)L.addends;
     p.box_bytes = (uint32_t)(kBoxN * g.bk * 2);
-    p.stage_bytes = p.entry_bytes + nt * p.box_bytes;
+    const uint32_t block_bytes = p.entry_bytes + nt * p.box_bytes;     // one kept block: weight tile (+ metadata) and X tile
     // Shared memory (the whole 227 KB; the base is 1024-aligned): the ring gets as many stages as fit next
     // to one staging tile per epilogue warp; what is left goes to the walk-list copy and to more staging
     // tiles.  Short walks are store-heavy and need no deep ring: they give stages up for staging tiles.
@@ -1073,8 +1215,23 @@ cudaError_t make_plan(const crisp_handle_s *h, int kind, const uint16_t *d_x, in
     const uint32_t epi = short_walk && nt >= 3 ? 4u * (uint32_t)nt : 8u;
     const bool nhwc = conv && conv->nhwc_out;                // transposed chunks need whole 4096-byte staging tiles
     const uint32_t fixed = epi * (nhwc ? 2 * kWideStageBytes : kWideStageBytes) + 256;
+    // Blocks per pipeline stage.  A stage costs each single-thread role (weight producer, X producer, MMA issuer)
+    // a fixed 300 to 400 cycles of waits, barrier arrivals and loop overhead on top of its copies and MMAs, which
+    // for short or narrow blocks is more than the tensor core needs for the block.  Where the ring still holds at
+    // least three of them, a stage therefore takes two or four consecutive walk entries: one weight-tile copy, one
+    // wait and one commit for all of them.  (Needs the tiled weight map; 256-column tiles of 64-deep blocks stay
+    // at one block per stage, two would leave room for two stages only.)
+    uint32_t group = 1;
+    const bool bounded = h->group_override > 0;        // a caller's bound: the largest feasible size below it
+    for (uint32_t g = 4; g >= 2; g >>= 1) {
+        if (bounded ? (int)g > h->group_override : L.wcap < 16) continue;   // walks below 16 blocks gain nothing (measured)
+        if ((g * p.entry_bytes) % 256 != 0 || (g * p.entry_bytes) / 256 > 256) continue;   // one box of the weight map
+        if ((avail - fixed) / (g * block_bytes) >= 3) { group = g; break; }
+    }
+    p.group = group;
+    p.stage_bytes = group * block_bytes;
     uint32_t stages = (avail - fixed) / p.stage_bytes;
-    const uint32_t max_stages = p.stage_bytes <= 24 * 1024 ? (wlen <= 8 ? 6u : 7u) : (wlen <= 8 ? 4u : 8u);
+    const uint32_t max_stages = block_bytes <= 24 * 1024 ? (wlen <= 8 ? 6u : 7u) : (wlen <= 8 ? 4u : 8u);
     if (stages > max_stages) stages = max_stages;
     if (stages < 2) return cudaErrorInvalidValue;
     p.num_stages = stages;
@@ -1092,8 +1249,11 @@ cudaError_t make_plan(const crisp_handle_s *h, int kind, const uint16_t *d_x, in
                  (p.walk_cache ? cache_bytes : 0);
 
     CUtensorMap &mx = plan->mx, &my = plan->my, &ma = plan->ma;
-    p.a_map = make_map_image(&ma, p.image, (uint64_t)L.stack * L.nst * L.wcap * L.entry_bytes, L.entry_bytes);
-    if (!p.a_map) ma = CUtensorMap{};
+    p.a_map = make_map_image(&ma, p.image, (uint64_t)L.stack * L.nst * L.wcap * L.entry_bytes, group * L.entry_bytes);
+    if (!p.a_map) {
+        if (group > 1) return cudaErrorInvalidValue;         // excluded above: a box of `group` entries fits the map's limits
+        ma = CUtensorMap{};
+    }
     const bool f32 = y_dtype != 0;
     p.stg_swz_mask = 7;
     if (conv) {
@@ -1177,6 +1337,7 @@ cudaError_t make_plan(const crisp_handle_s *h, int kind, const uint16_t *d_x, in
     info.stages = (int)stages;
     info.ctas = plan->grid;
     info.conv = conv ? 1 : 0;
+    info.stage_blocks = (int)p.group;
     return prepare_variant(plan->variant, device, plan->smem);
 }
 
@@ -1191,6 +1352,7 @@ cudaError_t launch_spmm_tc(crisp_handle_s *h, int kind, const uint16_t *d_x, int
     const bool hit = plan && plan->x == d_x && plan->y == d_y && plan->ldx == ldx && plan->ldy == ldy &&
                      plan->ncols == ncols && plan->y_dtype == y_dtype && plan->bias == h->epilogue.bias &&
                      plan->relu == h->epilogue.relu && plan->nt_override == h->nt_override &&
+                     plan->group_override == h->group_override &&
                      plan->device == device && plan->skip_stage == h->debug_skip_stage &&
                      plan->wait_limit == h->wait_limit_cycles && plan->has_conv == (conv != nullptr) &&
                      (!conv || same_conv(plan->conv, *conv)) && plan->p.status == h->d_status &&
@@ -1207,6 +1369,7 @@ cudaError_t launch_spmm_tc(crisp_handle_s *h, int kind, const uint16_t *d_x, int
         plan->x = d_x; plan->y = d_y; plan->bias = h->epilogue.bias;
         plan->ldx = ldx; plan->ldy = ldy; plan->ncols = ncols;
         plan->y_dtype = y_dtype; plan->relu = h->epilogue.relu; plan->nt_override = h->nt_override;
+        plan->group_override = h->group_override;
         plan->device = device; plan->skip_stage = h->debug_skip_stage; plan->wait_limit = h->wait_limit_cycles;
         plan->has_conv = conv != nullptr;
         if (conv) plan->conv = *conv;

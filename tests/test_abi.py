@@ -95,4 +95,5 @@ def test_handle_queries_reject_null(lib):
     info = B.LaunchInfo()
     assert lib.crisp_last_launch(None, C.byref(info)) == B.INVALID_ARG
     assert lib.crisp_set_tuning(None, 0, 0, -1) == B.INVALID_ARG
+    assert lib.crisp_set_stage_blocks(None, 0) == B.INVALID_ARG
     assert lib.crisp_reset_status(None, None) == B.INVALID_ARG

@@ -64,6 +64,26 @@ def test_conv_matches_oracle(env, s_out, kh, kw, pad, c, b, h, w, n, m, bm, keep
     L.close()
 
 
+def test_conv_blocks_per_stage_do_not_change_the_result(env):
+    """The gather with 1, 2 or 4 filter-tap blocks per pipeline stage: bit-identical outputs."""
+    B, torch = env
+    s_out, kh, kw, pad, c, b, h, w = 128, 3, 3, 1, 64, 2, 20, 24
+    wt, sal, act = conv_inputs(s_out, kh, kw, c, b, h, w, seed=77)
+    L = gpu_layer(B, torch, wt, sal, 2, 4, 64, 64, 0.6)
+    d_act = bf16_dev(act, torch)
+    ys = {}
+    for g in (1, 2, 4, 0):
+        L.set_stage_blocks(g)
+        y = L.spmm_conv(d_act, kh, kw, pad)
+        torch.cuda.synchronize()
+        assert L.device_status() == 0
+        assert 1 <= L.last_launch()["stage_blocks"] <= (g or 4)
+        ys[g] = y.clone()
+    for g in (2, 4, 0):
+        assert torch.equal(ys[1], ys[g]), g
+    L.close()
+
+
 def test_one_hot_taps_are_exact(env):
     """A weight with a single 1 per row picks shifted copies of the input: exact in bf16, border zeros included."""
     B, torch = env

@@ -294,7 +294,7 @@ def test_bounded_wait_reports_timeout_and_the_handle_stays_usable(env):
     mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
     L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
     d_x = bf16_dev(x, torch)
-    L.set_tuning(wait_limit_cycles=2_000_000, skip_fill=1)    # about a millisecond
+    L.set_tuning(wait_limit_cycles=2_000_000, skip_fill=0)    # about a millisecond; every CTA's first fill
     L.spmm(d_x)
     torch.cuda.synchronize()
     assert L.device_status() == B.TIMEOUT
@@ -304,6 +304,43 @@ def test_bounded_wait_reports_timeout_and_the_handle_stays_usable(env):
     torch.cuda.synchronize()
     assert L.device_status() == 0
     check_tolerance(y_to_f64(y, torch), oracle.spmm_fp64(wd, x))
+
+
+STAGE_CASES = [
+    (256, 1024, 1000, 2, 4, 32, 64, 0.5),             # union walks of odd length, ragged last column tile
+    (160, 960, 3136, 2, 8, 32, 32, 0.5),              # 32-deep blocks: up to four per stage
+    (512, 2304, 1536, 1, 4, 64, 64, 0.25),            # two row tiles per CTA tile
+    (128, 2048, 4096 + 64, 4, 8, 128, 64, 0.3),       # dense tiles, several tiles per CTA
+    (128, 1024, 640, 3, 4, 128, 64, 0.45),            # 3:4, dense tiles
+    (32, 64, 148 * 4 * 256 + 520, 2, 4, 32, 32, 1.0),  # stacked thin layer
+]
+
+
+@pytest.mark.parametrize("rows,k,ncols,n,m,bm,bk,keep", STAGE_CASES)
+def test_blocks_per_stage_do_not_change_the_result(env, rows, k, ncols, n, m, bm, bk, keep):
+    """A pipeline stage of 1, 2 or 4 kept blocks issues the same MMAs in the same order: the products are
+    bit-identical, walks that end inside a stage included, and equal to the oracle's within the tolerance."""
+    B, torch = env
+    w, s, x = rand_inputs(rows, k, ncols, seed=rows + k + ncols)
+    mk, vals, idx, wd, wb = oracle_layer(w, s, n, m, bm, bk, keep)
+    L = gpu_layer(B, torch, w, s, n, m, bm, bk, keep)
+    d_x = bf16_dev(x, torch)
+    ys, used = {}, {}
+    for g in (1, 2, 4, 0):
+        L.set_stage_blocks(g)
+        y = L.spmm(d_x)
+        torch.cuda.synchronize()
+        assert L.device_status() == 0
+        info = L.last_launch()
+        if info["path"] == B.PATH_DIRECT:
+            pytest.skip("direct kernel: no pipeline stages")
+        assert 1 <= info["stage_blocks"] <= (g or 4)
+        ys[g], used[g] = y.clone(), info["stage_blocks"]
+    assert used[1] == 1
+    for g in (2, 4, 0):
+        assert torch.equal(ys[1], ys[g]), (g, used)
+    check_tolerance(y_to_f64(ys[1], torch), oracle.spmm_fp64(wd, x))
+    L.close()
 
 
 def test_longest_row_of_blocks(env):
