@@ -200,16 +200,34 @@ group_bits_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec_
     }
 }
 
-// floor(v) of an fp32 value 0 <= v < 2^41 without a float-to-integer conversion per element (those run at a
-// fraction of the fp32 rate and were what bound this kernel): v = r + d with r = v rounded to a multiple of 2^20
-// (adding and subtracting 1.5 * 2^43 does that, exactly) and d = v - r exact, |d| <= 2^19; floor(d) by the same
-// device with 1.5 * 2^23 and a correction where it rounded up.  r and floor(d) are then added up in fp32 over the
-// eight elements of a row, which is exact (r / 2^20 <= 2^21 each, |floor(d)| <= 2^19 each), and converted once.
-__device__ __forceinline__ void floor_parts(float v, float &r, float &fd) {
-    r = __fsub_rn(__fadd_rn(v, 13194139533312.f), 13194139533312.f);            // 1.5 * 2^43
-    const float d = __fsub_rn(v, r);
-    const float t = __fsub_rn(__fadd_rn(d, 12582912.f), 12582912.f);            // 1.5 * 2^23: d to the nearest integer
-    fd = t > d ? __fsub_rn(t, 1.f) : t;
+// Two fp32 values in one 64-bit register and the packed fp32 instructions of sm_100 on them (one instruction
+// per pair; each half is rounded as the scalar instruction would round it).
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ float f32x2_sum(uint64_t v) {       // lo + hi
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return __fadd_rn(lo, hi);
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) { uint64_t r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) { uint64_t r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t add2_down(uint64_t a, uint64_t b) { uint64_t r; asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+
+// floor(v) of fp32 values 0 <= v < 2^41, two at a time, without a float-to-integer conversion per element (those
+// run at a fraction of the fp32 rate and were what bound this kernel): v = r + d with r = v rounded DOWN to a
+// multiple of 2^20 (add 1.5 * 2^43 rounding toward minus infinity: the sum lies in [2^43, 2^44), where fp32 steps
+// by 2^20; subtracting the constant again is exact) and d = v - r exact, 0 <= d < 2^20; floor(d) by the same device
+// with 1.5 * 2^23, where fp32 steps by 1.  r and floor(d) are then added up in fp32 over the eight elements of a
+// row, which is exact (r / 2^20 <= 2^21 each, floor(d) < 2^20 each), and converted once.
+__device__ __forceinline__ void floor_parts2(uint64_t v, uint64_t &r, uint64_t &fd) {
+    const uint64_t big = f32x2(13194139533312.f, 13194139533312.f);            // 1.5 * 2^43
+    const uint64_t mid = f32x2(12582912.f, 12582912.f);                        // 1.5 * 2^23
+    r = sub2(add2_down(v, big), big);
+    fd = sub2(add2_down(sub2(v, r), mid), mid);
 }
 
 // K-M1b: the block scores s_j = sum |T_w| as exact fixed-point integers, once the scale is known.  Second pass
@@ -245,14 +263,18 @@ block_score_kernel(const float *__restrict__ s, int64_t ld, Geometry g, bool vec
                 const int64_t row = x.row0 + warp * kM1RowsPerWarp + i;
                 uint32_t counted = 0xFFu;
                 if (g.score_mode == 0) counted = in_kp ? reinterpret_cast<const uint8_t *>(nm_bits + row * g.wpr)[k0 >> 3] : 0u;
-                float r_sum = 0.f, d_sum = 0.f;              // exact: see floor_parts
+                // an element that is not counted is multiplied by zero instead of by the scale: its parts are zero
+                uint64_t r_sum = f32x2(0.f, 0.f), d_sum = r_sum;             // exact: see floor_parts2
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float r, fd;
-                    floor_parts(__uint_as_float(key[i][j]) * scale, r, fd);
-                    if ((counted >> j) & 1u) { r_sum = __fadd_rn(r_sum, r); d_sum = __fadd_rn(d_sum, fd); }
+                for (int j = 0; j < 8; j += 2) {
+                    const uint64_t sc = f32x2((counted >> j) & 1u ? scale : 0.f, (counted >> (j + 1)) & 1u ? scale : 0.f);
+                    uint64_t r, fd;
+                    floor_parts2(mul2(f32x2(__uint_as_float(key[i][j]), __uint_as_float(key[i][j + 1])), sc), r, fd);
+                    r_sum = add2(r_sum, r);
+                    d_sum = add2(d_sum, fd);
                 }
-                acc += ((unsigned long long)__float2uint_rn(r_sum * 9.5367431640625e-07f) << 20) + (long long)__float2int_rn(d_sum);
+                acc += ((unsigned long long)__float2uint_rn(f32x2_sum(r_sum) * 9.5367431640625e-07f) << 20) +
+                       (unsigned long long)__float2uint_rn(f32x2_sum(d_sum));
             }
         } else {
 #pragma unroll
