@@ -968,7 +968,7 @@ def run_ours(args, layer, rank, world):
 
 
 def render_markdown(d):
-    """Markdown tables of one JSON line of this program (the tables of the benchmark spec are this output)."""
+    """Markdown tables of one JSON line of this program (the repository's table of measured numbers is this output)."""
     o = []
     r, ph, c = d["roofline"], d["phases"], d["config"]
     o.append(f"Headline step ({c['workload']}, {c['rows']}x{c['k']}x{c['ncols']}, block {c['block'][0]}x{c['block'][1]}, "
