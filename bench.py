@@ -655,6 +655,21 @@ def recorded_traffic(workload, kernel):
     return None
 
 
+def max_over_ranks(torch, value, world, device):
+    """The largest `value` over the ranks of the job: the slowest rank's time is the job's time."""
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank_step, world, ms_per_step):
+    """The path does not shard: N ranks are N replicas, each with the whole layer on its own inputs (weak scaling,
+    no data-path collective).  The job's throughput is all ranks' work over the slowest rank's step time."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 def run_ours(args, layer, rank, world):
     import torch
     import torch.distributed as dist
@@ -736,10 +751,7 @@ def run_ours(args, layer, rank, world):
     t_spmm = np.array([e[2].elapsed_time(e[3]) for e in ev])
     t_step = np.array([e[0].elapsed_time(e[3]) for e in ev])
     ms_local = float(t_step.sum() / args.steps)
-    ms_t = torch.tensor([ms_local], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
-    ms_per_step = float(ms_t.item())
+    ms_per_step = max_over_ranks(torch, ms_local, world, dev)
     status = L.device_status()
 
     # ---- dense bf16 cuBLAS GEMM of the same shape, same protocol
@@ -820,10 +832,7 @@ def run_ours(args, layer, rank, world):
     barrier()
     if not torch.equal(h_out[0], h_out[1]):
         raise SystemExit("end-to-end pipeline: the two result buffers differ")
-    e2e_ms = torch.tensor([a.elapsed_time(b) / e2e_steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_ms = float(e2e_ms.item())
+    e2e_ms = max_over_ranks(torch, a.elapsed_time(b) / e2e_steps, world, dev)
 
     # ---- end to end, inference style: the handle (mask + encoding) is reused, a step is X in -> product -> Y out.
     # Same pipelining: the copy of the next X and the read-back of the previous Y overlap the product.
@@ -857,10 +866,7 @@ def run_ours(args, layer, rank, world):
     inf_pipelined(e2e_steps, a)
     b.record(stream)
     barrier()
-    inf_ms = torch.tensor([a.elapsed_time(b) / e2e_steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(inf_ms, op=dist.ReduceOp.MAX)
-    inf_ms = float(inf_ms.item())
+    inf_ms = max_over_ranks(torch, a.elapsed_time(b) / e2e_steps, world, dev)
 
     # ---- the SpMM kernel as a stream of launches: back to back on three rotating sets of X / Y (384 MB, larger
     # than L2, so every launch finds its operands in HBM), one event pair around the whole stream
@@ -882,8 +888,8 @@ def run_ours(args, layer, rank, world):
     del xs, ys
 
     useful_flops = 2.0 * nnz * layer.ncols
-    value = world * useful_flops / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * useful_flops / (e2e_ms * 1e-3) / 1e12
+    value = whole_job_tflops(useful_flops, world, ms_per_step)
+    e2e_value = whole_job_tflops(useful_flops, world, e2e_ms)
 
     # ---- roofline of the dominant kernel (SpMM), from its live event time
     spmm_ms = float(t_spmm.mean())
@@ -937,7 +943,7 @@ def run_ours(args, layer, rank, world):
                    "overlap": "copies of step i+1 overlap compute and read-back of step i (2 buffer sets, 3 streams)",
                    "h2d_bytes_per_step": int(h_s.numel() * 4 + h_w.numel() * 2 + h_x.numel() * 2),
                    "d2h_bytes_per_step": int(h_y.numel() * 2)},
-           "e2e_inference": {"value": world * useful_flops / (inf_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": inf_ms,
+           "e2e_inference": {"value": whole_job_tflops(useful_flops, world, inf_ms), "unit": UNIT, "ms_per_step": inf_ms,
                              "step": "X host -> device, crisp_spmm on the resident handle, Y device -> host (2 buffer sets, 3 streams)",
                              "h2d_bytes_per_step": int(h_x.numel() * 2), "d2h_bytes_per_step": int(h_y.numel() * 2)},
            "gpu_launches": sum(kernels_per_step.values()) * args.steps, "kernels_per_step": kernels_per_step,

@@ -1,7 +1,8 @@
 """bench.py's CPU-only legs: the reference arm (the oracle timed on host cores) prints exactly one
 JSON line with the contract's keys, alone and under a 2-rank torchrun launch (rank 0 prints, the
 other rank exits 0 without work).  The path itself does not shard: N > 1 means independent replicas,
-so there is no collective to test beyond the launch and the single-line rule."""
+so the only exchange is the timed arm's maximum over the ranks' step times, which a two-rank gloo job checks
+together with the whole-job throughput formula."""
 import json
 import os
 import socket
@@ -47,3 +48,34 @@ def test_reference_arm_under_two_rank_torchrun():
                          cwd=ROOT, capture_output=True, text=True, timeout=900, env=env)
     assert out.returncode == 0, out.stderr[-2000:]
     _check_line(out.stdout, 2)
+
+
+def _aggregate_rank(rank, world, port, times_ms, flops, out):
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    try:
+        ms = bench.max_over_ranks(torch, times_ms[rank], world, torch.device("cpu"))
+        out[rank] = (ms, bench.whole_job_tflops(flops, world, ms))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_job_time_is_the_slowest_rank_and_value_counts_every_replica():
+    """The N > 1 path of the timed arm on two gloo ranks: every rank ends up with the maximum of the ranks' step
+    times, and the reported throughput is both replicas' work over that time."""
+    import torch.multiprocessing as mp
+    world, flops, times = 2, 3.0e12, [2.0, 5.0]
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_aggregate_rank, args=(world, _free_port(), times, flops, out), nprocs=world, join=True)
+        res = dict(out)
+    assert set(res) == {0, 1}
+    for ms, value in res.values():
+        assert ms == 5.0
+        assert abs(value - world * flops / 5.0e-3 / 1e12) < 1e-9
+    import bench, torch
+    assert bench.max_over_ranks(torch, 7.5, 1, torch.device("cpu")) == 7.5
+    assert bench.whole_job_tflops(1.0e12, 1, 1000.0) == 1.0
