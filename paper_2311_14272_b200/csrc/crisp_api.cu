@@ -220,7 +220,9 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     h->plan = nullptr;
     h->last = crisp_launch_info_t{-1, 0, 0, 1, 0, 0, 0, 0, 1};
     cudaStream_t st = (cudaStream_t)stream;
-    cudaError_t e = cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
+    // the status block is cleared by the encode kernel where one is launched with walk lists, else by a memset
+    const bool clear_in_kernel = h->exec_kind != CRISP_PATH_DIRECT && (int64_t)g.nrt * g.kkeep > 0;
+    cudaError_t e = clear_in_kernel ? cudaSuccess : cudaMemsetAsync(d_exec_buf, 0, kAlign, st);
     // 128-row blocks: one kept block is one tensor-core tile, so the encode kernel writes it directly
     const bool fuse_tiles = (h->exec_kind == CRISP_PATH_DENSE || h->exec_kind == CRISP_PATH_SPARSE) && g.bm == 128;
     crisp::TcImageLayout L = {};
@@ -229,6 +231,7 @@ crisp_status_t crisp_encode(const uint16_t *d_w_bf16, int64_t ld_w, crisp_mask_t
     const bool tc = h->exec_kind != CRISP_PATH_DIRECT;
     crisp::WalkArgs walks = {};
     if (tc) walks = crisp::tc_walk_args(g, h->exec_kind, mask->d_blk_col, h->d_exec);
+    walks.header = clear_in_kernel ? reinterpret_cast<uint32_t *>(d_exec_buf) : nullptr;
     if (e == cudaSuccess)
         e = crisp::launch_encode_canonical(d_w_bf16, ld_w, g, mask->d_blk_col, mask->d_nm_bits,
                                            h->d_blk_col, h->d_vals, h->d_idx, fuse_tiles ? h->exec_kind : 0,

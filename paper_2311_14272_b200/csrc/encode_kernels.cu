@@ -49,6 +49,7 @@ encode_block_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, bool
     extern __shared__ uint32_t s_buf[];
     // The first walks.nctas CTAs build the walk lists of the tensor-core kernel instead of encoding a block:
     // that needs only the mask's block list, so it overlaps the encoding instead of following it.
+    clear_header(walks);
     if ((int)blockIdx.x < walks.nctas) {
         __shared__ WalkShared s_walks;
         build_walks_body(g, walks, blockIdx.x, s_walks);
@@ -168,6 +169,7 @@ encode_block_m4_kernel(const uint16_t *__restrict__ w, int64_t ld, Geometry g, c
                        WalkArgs walks) {
     extern __shared__ uint32_t s_buf[];
     __shared__ uint32_t s_lut[16], s_lut_mask[16];
+    clear_header(walks);
     if ((int)blockIdx.x < walks.nctas) {
         __shared__ WalkShared s_walks;
         build_walks_body(g, walks, blockIdx.x, s_walks);

@@ -14,7 +14,14 @@ struct WalkArgs {
     int r, nst, wcap;
     int nctas;                    // CTAs that build walk lists (0: none), one per CTA tile
     int32_t *walk_col, *walk_len;
+    uint32_t *header = nullptr;   // 64 words that CTA 0 of the kernel clears (the handle's status block), or nullptr
 };
+
+// The status block at the head of the execution buffer, cleared by the kernel that fills the buffer: a memset of
+// its own in front of the kernel costs the stream about 2 us.
+__device__ __forceinline__ void clear_header(const WalkArgs &a) {
+    if (blockIdx.x == 0 && a.header != nullptr && threadIdx.x < 64) a.header[threadIdx.x] = 0u;
+}
 
 constexpr int kWalkBitmapWords = 128;                  // nblk <= 4096
 
