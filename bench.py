@@ -63,8 +63,8 @@ class ClockSampler:
     """Samples SM clock and throttle reasons while the timed region runs.
 
     NVML is read in-process (a sample costs microseconds, so even a timed region of a few milliseconds is
-    covered): by a thread every 0.5 ms and by `sample()` calls placed between steps (after a step has been queued in
-    full, never between the launches of a step: a slow host call there would let the GPU run dry mid-step).  Where NVML cannot
+    covered): by a thread every 0.5 ms and by `sample()` calls of the main thread while it waits for the queued steps
+    to finish (the timed steps are queued behind untimed work, so no launch waits for a host call).  Where NVML cannot
     be loaded, `nvidia-smi -lms` is read instead.  Reading only: no setting of the GPU is touched.
     """
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -731,6 +731,12 @@ def run_ours(args, layer, rank, world):
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
     barrier()
     sampler.start()
+    # The host must never be what a timed event pair waits for (a busy host, or this process's own sampling thread,
+    # can take longer to queue a launch than the GPU takes to run the previous one).  So some 15 ms of untimed fills
+    # go in first: while the GPU works through them the host queues every timed step, and the steps then run back
+    # to back off the stream's queue.
+    for _ in range(200):
+        flush.zero_()
     for i in range(args.steps):
         flush_l2()
         ev[i][0].record(stream)
@@ -740,10 +746,9 @@ def run_ours(args, layer, rank, world):
         ev[i][2].record(stream)
         L.spmm(d_x, y=d_y)
         ev[i][3].record(stream)
-        if i % 4 == 3:
-            sampler.sample()                       # between steps: step i is queued in full, so no launch of a
-                                                   # step waits for this host call
-    sampler.sample()                               # the stream is still busy with the steps queued above
+    while not ev[-1][3].query():                   # the sampling thread runs while the GPU works through the queue
+        sampler.sample()
+        time.sleep(0.0005)
     barrier()
     clocks = sampler.stop()
     t_mask = np.array([e[0].elapsed_time(e[1]) for e in ev])
@@ -755,17 +760,16 @@ def run_ours(args, layer, rank, world):
     status = L.device_status()
 
     # ---- dense bf16 cuBLAS GEMM of the same shape, same protocol
-    t_dense = []
-    for i in range(3 + args.steps):
+    evd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(3 + args.steps)]
+    for _ in range(100):                           # queued behind untimed fills, like the steps above
+        flush.zero_()
+    for a, b in evd:
         flush_l2()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         torch.matmul(d_w, d_x, out=d_y)
         b.record(stream)
-        torch.cuda.synchronize()
-        if i >= 3:
-            t_dense.append(a.elapsed_time(b))
-    t_dense = np.array(t_dense)
+    torch.cuda.synchronize()
+    t_dense = np.array([a.elapsed_time(b) for a, b in evd[3:]])
 
     # ---- end to end: pinned host inputs -> device, whole path, result back to pinned host memory.
     # Every step copies its own S, W and X from pinned host memory and its Y back; two sets of device
